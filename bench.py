@@ -78,8 +78,9 @@ def measured_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.period_s = period_s
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -115,7 +116,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.02)
+            time.sleep(self.period_s)
 
     def __enter__(self):
         if self._nv is not None:
@@ -145,12 +146,26 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+def config_block(workload_key, workloads):
+    """The ``config`` object of the JSON line: the same for the CUDA arm and for the reference (oracle) arm."""
+    from workload_flops import algorithmic_bytes
+    step_bytes = sum(algorithmic_bytes(w) for w in workloads)
+    flushed = step_bytes < (256 << 20)
+    return {"workload": workload_key, "variants": STEP_SETS[workload_key],
+            "shape": {k: getattr(workloads[0], k) for k in ("B", "Hq", "Hkv", "Sq", "Sk", "D")},
+            "l2": (f"inputs and outputs of a step ({step_bytes / 1e6:.0f} MB) are larger than the 126 MB L2; no flush"
+                   if not flushed else
+                   f"a step touches {step_bytes / 1e6:.1f} MB: L2 flushed (256 MB overwritten) before every launch; "
+                   "time = sum of the per-launch event intervals"),
+            "per_rank": "same workload on every GPU, different seeds, no collective"}, flushed
+
+
 def oracle_sample(workloads, target_rows):
     """Times the float64 oracle, as it stands, on evenly spaced rows of each variant.
     Returns (TFLOP/s over the unmasked FLOPs of those rows, threads, description, seconds)."""
     import oracle
     from oracle.attn_oracle import NORM_RELU, NORM_SIGMOID, NORM_SOFTMAX, OracleVariant
-    from paper_2605_05023_b200.flops import row_visibility
+    from workload_flops import row_visibility
 
     flops, secs, desc = 0.0, 0.0, []
     for w in workloads:
@@ -195,7 +210,7 @@ def run_reference(args, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * float(np.mean(secs)),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "variants": STEP_SETS[args.workload]},
+        "config": config_block(args.workload, workloads)[0],
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -373,7 +388,7 @@ def run_sweep(args):
     Appendix A variants this library builds.  Inputs are drawn on the device from a seeded generator; every
     point moves more than L2 (>= 270 MB); 3 warm-up and 20 timed launches per point, CUDA events."""
     import paper_2605_05023_b200 as pk
-    from paper_2605_05023_b200.flops import unmasked_flops
+    from workload_flops import unmasked_flops
     from synth_inputs import paper_sweep_workloads
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
@@ -424,6 +439,9 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=393216, help="oracle rows of the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 1.5 s steady-state run")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per-configuration roofline block")
+    ap.add_argument("--per-config-launches", type=int, default=60)
     ap.add_argument("--sweep", choices=["paper"], help="time the paper-shaped sweep instead (one JSON object; 1 GPU)")
     args = ap.parse_args()
     if args.sweep:
@@ -444,10 +462,27 @@ def main():
         run_reference(args, rank)
         return
 
+    run_attention(args, rank, world, local)
+
+
+# Variants whose kernel-only throughput the default line reports one by one (``roofline.per_config``): every large
+# bf16 configuration, each timed alone over back-to-back launches.
+PER_CONFIG_VARIANTS = ["c2_noncausal", "c2_causal", "c3_gqa_window_alibi", "c4a_softcap", "c4b_sigmoid", "c5_packed_doc_causal"]
+
+
+def kernel_name(w):
+    if w.dtype != "bf16":
+        return "attn_fwd_fp32_kernel"
+    if w.global_len is not None:
+        return "attn_fwd_split_kernel (one tile per CTA)"
+    return "attn_fwd_pair_kernel (CTA pairs)" if w.D == 256 else "attn_fwd_tc_kernel (two-tile ping-pong)"
+
+
+def run_attention(args, rank, world, local):
     args.warmup = max(args.warmup, 3)
     import torch.distributed as dist
     import paper_2605_05023_b200 as pk
-    from paper_2605_05023_b200.flops import algorithmic_bytes, unmasked_flops
+    from workload_flops import algorithmic_bytes, unmasked_flops
     from paper_2605_05023_b200.ranks import max_over_ranks, rank_seed, whole_job_throughput
 
     dev = torch.device(f"cuda:{local}")
@@ -464,23 +499,37 @@ def main():
     names = STEP_SETS[args.workload]
     workloads = [wl[n] for n in names]
     stream = torch.cuda.current_stream(dev)
+    peaks = measured_peaks()
+    gpu_index = physical_gpu_index(local)
 
-    # ---- resident inputs ----------------------------------------------------------------------
-    cases = []
-    for w in workloads:
+    def make_case(w):
         q, k, v = make_qkv(w.with_(seed=rank_seed(w.seed, rank)))   # every rank its own batch
         odt = torch.float32 if w.o_dtype == "fp32" else torch.bfloat16
-        c = {"w": w, "host": (q, k, v), "q": q.to(dev), "k": k.to(dev), "v": v.to(dev),
-             "o": torch.empty((w.B, w.Hq, w.Sq, w.D), device=dev, dtype=odt),
-             "lse": None if w.normalizer != "softmax" else torch.empty((w.B, w.Hq, w.Sq), device=dev, dtype=torch.float32),
-             "kw": pk.variant_kwargs(w, dev), "flops": unmasked_flops(w), "bytes": algorithmic_bytes(w),
-             "status": torch.zeros(64, dtype=torch.int32, device=dev)}
-        cases.append(c)
+        return {"w": w, "host": (q, k, v), "q": q.to(dev), "k": k.to(dev), "v": v.to(dev),
+                "o": torch.empty((w.B, w.Hq, w.Sq, w.D), device=dev, dtype=odt),
+                "lse": None if w.normalizer != "softmax" else torch.empty((w.B, w.Hq, w.Sq), device=dev, dtype=torch.float32),
+                "kw": pk.variant_kwargs(w, dev), "flops": unmasked_flops(w), "bytes": algorithmic_bytes(w),
+                "status": torch.zeros(1, dtype=torch.int32, device=dev)}
+
+    def launch(c):
+        pk.attn_fwd(c["q"], c["k"], c["v"], o=c["o"], lse=c["lse"], stream=stream, status_word=c["status"], **c["kw"])
+
+    def status_error(cs):
+        bad = None
+        for c in cs:
+            word = int(c["status"].item())
+            if word != 0:
+                bad = f"{c['w'].name}: kernel reported status {word} ({pk.status_string(word)})"
+                c["status"].zero_()
+        return bad
+
+    # ---- resident inputs ----------------------------------------------------------------------
+    cases = [make_case(w) for w in workloads]
     step_flops = float(sum(c["flops"] for c in cases))
     # A step whose inputs and outputs fit in L2 (126 MB) gets the L2 flushed before every launch (a 256 MB
     # buffer is overwritten); its time is then the sum of the per-launch CUDA-event intervals.
-    step_bytes = sum(c["bytes"] for c in cases)
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if step_bytes < (256 << 20) else None
+    config, flushed = config_block(args.workload, workloads)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if flushed else None
 
     def step(events=None):
         for c in cases:
@@ -489,7 +538,7 @@ def main():
             if events is not None:
                 e0 = torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-            pk.attn_fwd(c["q"], c["k"], c["v"], o=c["o"], lse=c["lse"], stream=stream, status_word=c["status"], **c["kw"])
+            launch(c)
             if events is not None:
                 e1 = torch.cuda.Event(enable_timing=True)
                 e1.record(stream)
@@ -506,19 +555,14 @@ def main():
         kernel_events = []
         t_start = torch.cuda.Event(enable_timing=True)
         t_stop = torch.cuda.Event(enable_timing=True)
-        with ClockSampler(physical_gpu_index(local)) as clocks:
+        with ClockSampler(gpu_index, period_s=0.001) as clocks:
             t_start.record(stream)
             for _ in range(args.steps):
                 step(kernel_events)
             t_stop.record(stream)
             barrier()
         launches = pk.launch_count() - launches0
-        bad = None
-        for c in cases:
-            words = c["status"].cpu().tolist()     # word 0 is the status; debug builds of the library fill the rest
-            if words[0] != 0:
-                bad = f"{c['w'].name}: kernel reported status {words[0]} ({pk.status_string(words[0])}); status words: {words}"
-                c["status"].zero_()
+        bad = status_error(cases)
         if world > 1:   # every rank repeats if any rank has to
             flag = torch.tensor([1 if bad else 0], device=dev)
             dist.all_reduce(flag, op=dist.ReduceOp.MAX)
@@ -535,6 +579,7 @@ def main():
         ms_total = float(sum(e0.elapsed_time(e1) for _, e0, e1 in kernel_events))
     ms_total = max_over_ranks(ms_total, dev)
     value = whole_job_throughput(step_flops * args.steps, ms_total * 1e-3, world) / 1e12
+    clock_summary = clocks.summary()
 
     # per-kernel durations (CUDA events on the launching stream), for the roofline
     per_variant = {}
@@ -542,25 +587,25 @@ def main():
         per_variant.setdefault(name, []).append(e0.elapsed_time(e1))
     kernel_ms = sum(float(np.sum(v)) for v in per_variant.values())
     n_launch = sum(len(v) for v in per_variant.values())
-    peaks = measured_peaks()
     flops_per_launch = step_flops * args.steps / n_launch
     ms_per_launch = kernel_ms / n_launch
     compute_bound = workloads[0].dtype == "bf16"
+    traffic_note = "stored figure: dram__bytes_read.sum + dram__bytes_write.sum of one launch from the ncu captures under profiles/, not measured in this run"
     if compute_bound:
         achieved = flops_per_launch / (ms_per_launch * 1e-3) / 1e12
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "traffic": ncu_traffic(args.workload),
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": ncu_traffic(args.workload), "traffic_note": traffic_note,
                     "peak_kind": f"bf16 dense burst, of {peaks['source']}",
-                    "frac_of_sustained_peak": (achieved / peaks["bf16_tflops_sustained"]) if peaks["bf16_tflops_sustained"] else None,
-                    "kernel": "attn_fwd_pair_kernel (CTA pairs)" if workloads[0].D == 256 else "attn_fwd_tc_kernel (two-tile ping-pong)",
+                    "kernel": kernel_name(workloads[0]),
                     "launches": n_launch, "ms_per_launch": ms_per_launch,
+                    "ms_x_sm_mhz": (ms_per_launch * clock_summary["sm_mhz"]) if clock_summary["sm_mhz"] else None,
                     "median_ms_per_launch": {n: float(np.median(v)) for n, v in per_variant.items()},
                     "per_variant_tflops": {n: float(unmasked_flops(wl[n]) / (np.mean(v) * 1e-3) / 1e12)
                                            for n, v in per_variant.items()}}
     else:
         gbs = sum(c["bytes"] for c in cases) * args.steps / n_launch / (ms_per_launch * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                    "frac": gbs / peaks["hbm_gbs"], "traffic": ncu_traffic(args.workload),
+                    "frac": gbs / peaks["hbm_gbs"], "traffic": ncu_traffic(args.workload), "traffic_note": traffic_note,
                     "peak_kind": f"copy bandwidth, of {peaks['source']}; this workload (17 MFLOP, 0.5 MB) is launch-latency bound",
                     "kernel": "attn_fwd_fp32_kernel", "launches": n_launch, "ms_per_launch": ms_per_launch,
                     "median_ms_per_launch": {n: float(np.median(v)) for n, v in per_variant.items()}}
@@ -571,11 +616,35 @@ def main():
                 for c in cases:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record(stream)
-                    pk.attn_fwd(c["q"], c["k"], c["v"], o=c["o"], lse=c["lse"], stream=stream, status_word=c["status"], **c["kw"])
+                    launch(c)
                     e1.record(stream)
                     warm.append((e0, e1))
             torch.cuda.synchronize()
             roofline["warm_l2_median_ms_per_launch"] = float(np.median([a.elapsed_time(b) for a, b in warm]))
+
+    # ---- the same step repeated for at least 1.5 s: the power-capped steady state ------------------
+    # (A short timed region runs at the boost clock; a long one settles at the clock the 1000 W limit allows.  The
+    # contract value above is the K steps asked for; this block says what a long-running job sees.)
+    sustained = None
+    if compute_bound and world == 1 and not args.no_sustained:
+        n_sus = max(args.steps, int(np.ceil(1500.0 / max(ms_total / args.steps, 1e-3))))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(gpu_index, period_s=0.01) as sus_clocks:
+            s0.record(stream)
+            for _ in range(n_sus):
+                step()
+            s1.record(stream)
+            torch.cuda.synchronize()
+        bad = status_error(cases)
+        if bad is not None:
+            raise RuntimeError(bad)
+        ms_sus = s0.elapsed_time(s1)
+        v_sus = step_flops * n_sus / (ms_sus * 1e-3) / 1e12
+        sc = sus_clocks.summary()
+        sustained = {"value": v_sus, "unit": UNIT, "steps": n_sus, "seconds": ms_sus * 1e-3, "ms_per_step": ms_sus / n_sus,
+                     "clocks": sc, "ms_per_step_x_sm_mhz": (ms_sus / n_sus * sc["sm_mhz"]) if sc["sm_mhz"] else None,
+                     "frac_of_burst_peak": v_sus / peaks["bf16_tflops"],
+                     "frac_of_sustained_peak": (v_sus / peaks["bf16_tflops_sustained"]) if peaks["bf16_tflops_sustained"] else None}
 
     # ---- end to end: pinned host buffers through attn_fwd_host ------------------------------------
     e2e = None
@@ -635,6 +704,47 @@ def main():
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                "ms_per_step": ms_e2e / e2e_steps,
                "api": "attn_fwd_host (pinned host buffers, copies in the timed region; one stream per call of the step)"}
+        del hcases
+
+    # ---- every large configuration on its own (rank 0, N = 1 only) ---------------------------------
+    per_config = None
+    if compute_bound and rank == 0 and world == 1 and not args.no_per_config:
+        per_config = {}
+        by_name = {c["w"].name: c for c in cases}
+        n_pc = max(50, args.per_config_launches)
+        for name in PER_CONFIG_VARIANTS:
+            c = by_name.get(name) or make_case(wl[name])
+            for _ in range(5):
+                launch(c)
+            torch.cuda.synchronize()
+            evs = []
+            with ClockSampler(gpu_index) as pc_clocks:
+                for _ in range(n_pc):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    launch(c)
+                    e1.record(stream)
+                    evs.append((e0, e1))
+                torch.cuda.synchronize()
+            bad = status_error([c])
+            if bad is not None:
+                raise RuntimeError(bad)
+            ms = np.array([a.elapsed_time(b) for a, b in evs])
+            pc = pc_clocks.summary()
+            tf = c["flops"] / (float(ms.mean()) * 1e-3) / 1e12
+            per_config[name] = {
+                "flops_per_launch": float(c["flops"]), "launches": n_pc, "mean_ms": float(ms.mean()), "median_ms": float(np.median(ms)),
+                "tflops": tf, "tflops_at_median": c["flops"] / (float(np.median(ms)) * 1e-3) / 1e12,
+                "frac_of_burst_peak": tf / peaks["bf16_tflops"], "algorithmic_bytes": int(c["bytes"]),
+                "traffic": NCU_TRAFFIC_BYTES_PER_VARIANT.get(name), "kernel": kernel_name(c["w"]),
+                "sm_mhz": pc["sm_mhz"], "clock_samples": pc["samples"], "reasons": pc["reasons"],
+                "mean_ms_x_sm_mhz": (float(ms.mean()) * pc["sm_mhz"]) if pc["sm_mhz"] else None}
+            if name not in by_name:
+                del c
+                torch.cuda.empty_cache()
+        roofline["per_config"] = per_config
+        roofline["per_config_note"] = (f"each configuration alone, {n_pc} back-to-back launches after 5 warm-up launches, CUDA events per launch; "
+                                       "inputs and outputs of every configuration exceed L2; traffic = stored ncu figures")
 
     # ---- oracle on the host cores (rank 0, N = 1 only) -------------------------------------------
     cpu = None
@@ -643,20 +753,13 @@ def main():
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": secs}
 
     if rank == 0:
-        in_bytes = sum(c["bytes"] for c in cases)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if compute_bound else "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "variants": names,
-                       "shape": {k: getattr(workloads[0], k) for k in ("B", "Hq", "Hkv", "Sq", "Sk", "D")},
-                       "l2": (f"inputs and outputs of a step ({in_bytes / 1e6:.0f} MB) are larger than the 126 MB L2; no flush"
-                              if flush_buf is None else
-                              f"a step touches {in_bytes / 1e6:.1f} MB: L2 flushed (256 MB overwritten) before every launch; "
-                              "time = sum of the per-launch event intervals"),
-                       "per_rank": "same workload on every GPU, different seeds, no collective"},
+            "config": config,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks.summary(), "rejected_runs": rejected,
+            "clocks": clock_summary, "sustained": sustained, "rejected_runs": rejected,
             "pct_of_nominal_dense_bf16_peak": 100.0 * value / world / 2250.0,
         }
         print(json.dumps(line), flush=True)

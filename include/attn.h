@@ -35,7 +35,11 @@
  *     the caller; the descriptor itself is HOST memory, read during the call only.
  *   - The call enqueues work on `stream` and returns; it never synchronises, never prints
  *     and never aborts.  Device arrays must stay valid until the stream work is done.
- *   - Any failure is a non-zero attn_status return with nothing launched.
+ *   - Any failure is a non-zero attn_status return; every argument check runs before the first CUDA call, so an
+ *     argument error leaves nothing on the stream (attn_fwd_host included: no copy is enqueued either).
+ *   - Thread safety: every entry point may be called from several host threads at once, on the same or on
+ *     different devices (the per-device set-up of the first call and the tensor-map cache are guarded); calls
+ *     that share a stream are ordered by CUDA as usual.
  *   - Layout: q, o are [B, Hq, Sq, D]; k, v are [B, Hkv, Sk, D]; lse is [B, Hq, Sq] fp32,
  *     contiguous.  Strides (in elements, for batch / head / row) may be given in the
  *     descriptor; all-zero means contiguous.  The innermost dimension is always dense.
@@ -98,8 +102,10 @@ typedef struct attn_variant_desc {
     int64_t  k_strides[3];
     int64_t  v_strides[3];
     int64_t  o_strides[3];
-    int32_t* status_word;      /* optional device int32: a kernel that gives up a bounded wait stores
-                                  ATTN_ERR_TIMEOUT here (never cleared by the library) */
+    int32_t* status_word;      /* optional device int32, zeroed by the caller (the library never clears it): a kernel
+                                  that gives up a bounded wait stores ATTN_ERR_TIMEOUT here; a cu_seqlens table that
+                                  does not start at 0, end at Sq or that decreases somewhere is reported as
+                                  ATTN_ERR_DESC (the kernel stays memory safe and the output is unspecified) */
 } attn_variant_desc;
 
 /*
@@ -119,7 +125,7 @@ typedef struct attn_variant_desc {
  * B == 1 and Sq == Sk.
  *
  * The first call on a device loads the kernels and sets their shared-memory attribute.
- * Returns ATTN_OK or an attn_status; on error nothing was launched.
+ * Returns ATTN_OK or an attn_status; on an argument error nothing was launched.
  */
 int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
              int B, int Hq, int Hkv, int Sq, int Sk, int D,
@@ -155,6 +161,30 @@ int attn_version(void);
 
 /* Number of kernel launches attn_fwd has issued in this process (for benchmarks). */
 int64_t attn_launch_count(void);
+
+/*
+ * attn_clear_cache -- empties the library's cache of encoded TMA tensor maps (host memory only).  The tensor-core
+ * kernels read Q, K and V tiles (Eq. 1) through tensor maps, which are pure functions of (base address, shape,
+ * strides, box); a call on tensors seen before reuses the cached encoding.  An entry is never stale, so clearing
+ * is never needed for correctness; it returns the table to its initial state.  Always ATTN_OK.
+ */
+int attn_clear_cache(void);
+
+/* Number of tensor-map look-ups served from that cache in this process (for tests and benchmarks). */
+int64_t attn_cache_hits(void);
+
+/*
+ * attn_selftest_timeout -- exercises the failure path of the kernels' bounded waits without a fault: launches
+ * a one-CTA kernel in which one thread waits, for at most limit_ns, on an mbarrier that nothing arrives on (the
+ * kernels that compute Eq. 1 / Eq. 2 link their roles with such barriers).  When the limit passes it stores
+ * ATTN_ERR_TIMEOUT in *status_word and raises the CTA's abort flag; a second thread waiting on the same barrier
+ * with the kernels' full limit sees the flag and returns at once (it stores 2 in *second_waiter, if given);
+ * the kernel ends normally and the context stays usable.
+ *
+ *   status_word    device int32, zeroed by the caller.       second_waiter   device int32 or NULL.
+ *   limit_ns       1 .. 100 000 000 (0.1 s); outside: ATTN_ERR_DESC, nothing launched.
+ */
+int attn_selftest_timeout(int32_t* status_word, uint64_t limit_ns, int32_t* second_waiter, void* stream);
 
 #ifdef __cplusplus
 }

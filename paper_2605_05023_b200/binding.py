@@ -74,6 +74,10 @@ _lib.attn_status_string.restype = ctypes.c_char_p
 _lib.attn_status_string.argtypes = [ctypes.c_int]
 _lib.attn_version.restype = ctypes.c_int
 _lib.attn_launch_count.restype = ctypes.c_int64
+_lib.attn_clear_cache.restype = ctypes.c_int
+_lib.attn_cache_hits.restype = ctypes.c_int64
+_lib.attn_selftest_timeout.restype = ctypes.c_int
+_lib.attn_selftest_timeout.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p]
 
 
 def status_string(status: int) -> str:
@@ -86,6 +90,23 @@ def version() -> int:
 
 def launch_count() -> int:
     return int(_lib.attn_launch_count())
+
+
+def clear_cache() -> int:
+    """``attn_clear_cache``: empties the cache of encoded tensor maps."""
+    return int(_lib.attn_clear_cache())
+
+
+def cache_hits() -> int:
+    return int(_lib.attn_cache_hits())
+
+
+def selftest_timeout(status_word: torch.Tensor, limit_ns: int, second_waiter: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> int:
+    """``attn_selftest_timeout``: one bounded wait that runs out, on purpose; returns the attn_status of the launch."""
+    st = stream if stream is not None else torch.cuda.current_stream(status_word.device)
+    return int(_lib.attn_selftest_timeout(status_word.data_ptr(), int(limit_ns),
+                                          second_waiter.data_ptr() if second_waiter is not None else None, st.cuda_stream))
 
 
 def raw_attn_fwd(q_ptr, k_ptr, v_ptr, o_ptr, lse_ptr, B, Hq, Hkv, Sq, Sk, D,

@@ -1,18 +1,74 @@
-// Host side of the C ABI declared in include/attn.h: argument validation, parameter
-// block, kernel selection.  Nothing here computes; every step of the path runs in the
-// kernels of attn_simt_fp32.cu (fp32 inputs) and attn_tc_bf16.cu (bf16 inputs, tcgen05).
+// Host side of the C ABI declared in include/attn.h: argument validation, parameter block, kernel selection,
+// and the cache of encoded TMA tensor maps.  Nothing here computes; every step of the path runs in the kernels
+// of attn_simt_fp32.cu (fp32 inputs) and attn_tc_pingpong.cu / attn_tc_pair.cu / attn_tc_split.cu (bf16 inputs,
+// tcgen05).
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/attn.h"
 #include "attn_params.cuh"
+#include "attn_tc_common.cuh"
 
 namespace b200attn {
 cudaError_t launch_attn_fwd_fp32(const AttnParams& p, cudaStream_t stream);
 // Returns ATTN_OK, ATTN_ERR_UNSUPPORTED or ATTN_ERR_CUDA; *launches receives the number of
 // kernels enqueued.
 int launch_attn_fwd_bf16(const AttnParams& p, cudaStream_t stream, int* launches);
+}  // namespace b200attn
+
+namespace b200attn {
+namespace tc {
+
+// Encoded tensor maps are pure functions of (address, shape, strides, box): they are kept in a small direct-mapped
+// table so that a call on tensors seen before skips the driver's encoder.  One mutex guards the table; an entry is
+// never stale (the same key always encodes to the same 128 bytes), attn_clear_cache() merely empties it.
+namespace {
+constexpr int kMapCacheSlots = 256;
+struct MapSlot { bool used; MapKey key; CUtensorMap map; };
+MapSlot g_map_cache[kMapCacheSlots];
+std::mutex g_map_mutex;
+std::atomic<long long> g_map_hits{0};
+
+bool same_key(const MapKey& a, const MapKey& b) {
+    return a.ptr == b.ptr && a.B == b.B && a.H == b.H && a.S == b.S && a.D == b.D && a.st[0] == b.st[0] &&
+           a.st[1] == b.st[1] && a.st[2] == b.st[2] && a.box_rows == b.box_rows && a.box_cols == b.box_cols;
+}
+size_t slot_of(const MapKey& k) {
+    uint64_t h = reinterpret_cast<uintptr_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
+    h ^= ((uint64_t)k.S << 32) ^ ((uint64_t)k.H << 16) ^ ((uint64_t)k.B << 8) ^ (uint64_t)k.D ^ ((uint64_t)k.box_rows << 48) ^
+         ((uint64_t)k.box_cols << 56) ^ ((uint64_t)k.st[2] * 0xC2B2AE3D27D4EB4Full);
+    return (size_t)((h >> 29) % kMapCacheSlots);
+}
+}  // namespace
+
+bool cached_map(CUtensorMap* out, const MapKey& key) {
+    MapSlot& slot = g_map_cache[slot_of(key)];
+    {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        if (slot.used && same_key(slot.key, key)) {
+            *out = slot.map;
+            g_map_hits.fetch_add(1, std::memory_order_relaxed);
+            return true;
+        }
+    }
+    if (!encode_map(out, key)) return false;
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    slot.used = true;
+    slot.key = key;
+    slot.map = *out;
+    return true;
+}
+
+void clear_map_cache() {
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    for (MapSlot& s : g_map_cache) s.used = false;
+}
+
+long long map_cache_hits() { return g_map_hits.load(std::memory_order_relaxed); }
+
+}  // namespace tc
 }  // namespace b200attn
 
 namespace {
@@ -40,31 +96,11 @@ bool resolve_strides(const int64_t in[3], long long out[3], int H, int S, int D,
     return true;
 }
 
-}  // namespace
 
-extern "C" {
-
-const char* attn_status_string(int status) {
-    switch (status) {
-        case ATTN_OK: return "ok";
-        case ATTN_ERR_NULL: return "a required pointer is NULL";
-        case ATTN_ERR_SHAPE: return "invalid shape";
-        case ATTN_ERR_UNSUPPORTED: return "unsupported dtype, head dimension or combination";
-        case ATTN_ERR_ALIGN: return "pointer or stride is not 16-byte aligned";
-        case ATTN_ERR_DESC: return "malformed variant descriptor";
-        case ATTN_ERR_CUDA: return "a CUDA call failed";
-        case ATTN_ERR_TIMEOUT: return "a bounded device-side wait gave up";
-        default: return "unknown status";
-    }
-}
-
-int attn_version(void) { return 100; }
-
-int64_t attn_launch_count(void) { return g_launches.load(); }
-
-int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
-             int B, int Hq, int Hkv, int Sq, int Sk, int D,
-             const attn_variant_desc* desc, void* stream) {
+// Every argument check of attn_fwd, made before any CUDA call; fills the kernels' parameter block.
+int check_and_fill(const void* q, const void* k, const void* v, void* o, float* lse,
+                   int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                   const attn_variant_desc* desc, b200attn::AttnParams* out) {
     using namespace b200attn;
     if (!q || !k || !v || !o || !desc) return ATTN_ERR_NULL;
     if (desc->struct_size != sizeof(attn_variant_desc)) return ATTN_ERR_DESC;
@@ -133,9 +169,15 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
     p.normalizer = (int)desc->normalizer;
     p.o_fp32 = desc->o_dtype == ATTN_FP32;
     p.status_word = desc->status_word;
+    *out = p;
+    return ATTN_OK;
+}
 
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (desc->dtype == ATTN_FP32) {
+
+// Kernel selection and launch for a checked parameter block.
+int launch_checked(const b200attn::AttnParams& p, uint32_t dtype, cudaStream_t st) {
+    using namespace b200attn;
+    if (dtype == ATTN_FP32) {
         if (launch_attn_fwd_fp32(p, st) != cudaSuccess) return ATTN_ERR_CUDA;
         g_launches.fetch_add(1);
         return ATTN_OK;
@@ -145,6 +187,43 @@ int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
     g_launches.fetch_add(launches);
     return rc;
 }
+
+}  // namespace
+
+extern "C" {
+
+const char* attn_status_string(int status) {
+    switch (status) {
+        case ATTN_OK: return "ok";
+        case ATTN_ERR_NULL: return "a required pointer is NULL";
+        case ATTN_ERR_SHAPE: return "invalid shape";
+        case ATTN_ERR_UNSUPPORTED: return "unsupported dtype, head dimension or combination";
+        case ATTN_ERR_ALIGN: return "pointer or stride is not 16-byte aligned";
+        case ATTN_ERR_DESC: return "malformed variant descriptor";
+        case ATTN_ERR_CUDA: return "a CUDA call failed";
+        case ATTN_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+int attn_version(void) { return 100; }
+
+int64_t attn_launch_count(void) { return g_launches.load(); }
+
+int attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+             int B, int Hq, int Hkv, int Sq, int Sk, int D,
+             const attn_variant_desc* desc, void* stream) {
+    b200attn::AttnParams p;
+    if (const int rc = check_and_fill(q, k, v, o, lse, B, Hq, Hkv, Sq, Sk, D, desc, &p)) return rc;
+    return launch_checked(p, desc->dtype, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int attn_clear_cache(void) {
+    b200attn::tc::clear_map_cache();
+    return ATTN_OK;
+}
+
+int64_t attn_cache_hits(void) { return b200attn::tc::map_cache_hits(); }
 
 namespace {
 size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -185,12 +264,16 @@ int attn_fwd_host(const void* q_host, const void* k_host, const void* v_host, vo
     char* ws = static_cast<char*>(workspace);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const bool want_lse = lse_host && desc->normalizer == ATTN_NORM_SOFTMAX;
+    // Every argument check runs before the first copy is enqueued: on an argument error nothing reaches the stream.
+    b200attn::AttnParams p;
+    if (const int rc = check_and_fill(ws + L.q, ws + L.k, ws + L.v, ws + L.o, want_lse ? reinterpret_cast<float*>(ws + L.lse) : nullptr,
+                                      B, Hq, Hkv, Sq, Sk, D, desc, &p))
+        return rc;
     if (cudaMemcpyAsync(ws + L.q, q_host, L.qb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(ws + L.k, k_host, L.kvb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(ws + L.v, v_host, L.kvb, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return ATTN_ERR_CUDA;
-    const int rc = attn_fwd(ws + L.q, ws + L.k, ws + L.v, ws + L.o, want_lse ? reinterpret_cast<float*>(ws + L.lse) : nullptr,
-                            B, Hq, Hkv, Sq, Sk, D, desc, stream);
+    const int rc = launch_checked(p, desc->dtype, st);
     if (rc != ATTN_OK) return rc;
     if (cudaMemcpyAsync(o_host, ws + L.o, L.ob, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ATTN_ERR_CUDA;
     if (want_lse && cudaMemcpyAsync(lse_host, ws + L.lse, L.lseb, cudaMemcpyDeviceToHost, st) != cudaSuccess)

@@ -66,7 +66,9 @@ __device__ __forceinline__ RowInterval row_interval(const AttnParams& p, int i, 
     const int ip = i + p.Sk - p.Sq;
     int lo = 0, hi = p.Sk - 1, doc = 0;
     if (p.mask_flags & kMaskCausal) hi = min(hi, max(ip, p.prefix_len - 1));
-    if (ip < p.global_len) return RowInterval{0, hi, 0, 0};      // a global token's row: only the causal clause
+    // A global token's row keeps only the causal clause.  (Tested on the flag: with Sq > Sk a row has i' < 0, which
+    // is below global_len = 0 of a call without global tokens.)
+    if ((p.mask_flags & kMaskGlobal) && ip < p.global_len) return RowInterval{0, hi, 0, 0};
     if (p.mask_flags & kMaskWindow) {
         if (p.window_left >= 0) lo = max(lo, ip - p.window_left);
         if (p.window_right >= 0) hi = min(hi, ip + p.window_right);
@@ -78,7 +80,7 @@ __device__ __forceinline__ RowInterval row_interval(const AttnParams& p, int i, 
     }
     // Global tokens as keys: [0, global_len) joins the interval when they touch, else it is a second piece.
     int pre = 0;
-    if (p.global_len > 0) {
+    if (p.mask_flags & kMaskGlobal) {
         if (lo > hi) { lo = 0; hi = p.global_len - 1; }          // (the causal clause holds: global_len <= i')
         else if (lo <= p.global_len) { lo = 0; hi = max(hi, p.global_len - 1); }
         else pre = p.global_len;
@@ -113,7 +115,7 @@ __device__ __forceinline__ TileBounds tile_bounds(const AttnParams& p, int q0, i
         t.lo_max = max(t.lo_max, row_interval(p, p.test_query_start - 1).lo);
     t.pre_min = min(a.pre, b.pre);
     t.pre_max = max(a.pre, b.pre);
-    if (p.global_len > 0) {
+    if (p.mask_flags & kMaskGlobal) {
         // Rows of global tokens see up to the causal bound, the others up to their window: hi is not monotone
         // across position global_len, and with a test query the prefix piece is not either.  A tile that holds
         // such a break takes the union of its ends and classifies no key tile as fully visible.

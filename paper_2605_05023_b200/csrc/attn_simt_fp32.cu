@@ -17,6 +17,7 @@
 // why staged rows past Sk are zero-filled.  The kernel is compiled per number of 32-column
 // groups of the head dimension.
 #include "attn_params.cuh"
+#include "sm100_sync.cuh"
 
 namespace b200attn {
 
@@ -57,6 +58,8 @@ attn_fwd_fp32_kernel(const AttnParams p) {
     float* q_sm = simt_smem;                                   // [kSimtWarps][D]
     float* kv_sm = simt_smem + kSimtWarps * D;                 // [kSimtStages][K | V][32][ld]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (blockIdx.x == 0 && warp == 0 && (p.mask_flags & kMaskDocument))
+        tc::check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);
 
     const int nrb = (p.Sq + kSimtWarps - 1) / kSimtWarps;      // row blocks per (batch, head)
     const int rb = blockIdx.x % nrb;

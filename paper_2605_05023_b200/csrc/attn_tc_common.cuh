@@ -1,18 +1,21 @@
 // Pieces shared by the three tensor-core attention kernels (attn_tc_pingpong.cu, attn_tc_pair.cu,
-// attn_tc_split.cu): tile sizes and constants, the tcgen05 instruction descriptor, the exponential step of the
-// online softmax, the warp-level arrival after TMEM stores, and the host-side TMA tensor maps.
+// attn_tc_split.cu): tile sizes and constants, the tcgen05 instruction descriptor, the element-wise mask of a
+// partial tile, the exponential step of the online softmax, and the host-side TMA tensor maps.  (Bounded waits,
+// the work-item fetch and the warp-level arrivals are in sm100_sync.cuh.)
 #pragma once
+#include <atomic>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "sm100_ptx.cuh"
+#include "sm100_sync.cuh"
 
 namespace b200attn {
 namespace tc {
 
 constexpr int kBM = 128;                         // query rows per tile
 constexpr int kBN = 128;                         // keys per tile
-constexpr uint64_t kWaitLimitNs = 2000000000ull; // bounded waits give up after 2 s
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^8
@@ -27,17 +30,23 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// One arrival per warp: the warp converges first, so that every lane's earlier shared-memory / TMEM traffic is
-// ordered before the arrival (the barriers count one arrival per softmax warp).
-__device__ __forceinline__ void warp_arrive(uint32_t bar) {
-    __syncwarp();
-    if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(bar);
+// Mask of a partial tile (Appendix A.2; loop splitting, Sec. 3.4: only tiles that straddle an edge of a row's
+// interval come here).  y holds 32 score columns of one row; columns outside [a, e] (chunk-relative, inclusive)
+// become -inf.  Two forms with the same result: one bit test per element against a visibility word built with
+// two shifts, or two compares per element (a few kernel instances are faster with the latter).
+// `pre` adds a second visible piece: the columns below it (global tokens; 0 = none).
+__device__ __forceinline__ void mask_chunk32_bits(uint32_t* y, int a, int e, int pre = 0) {
+    const int lo = max(a, 0), hi = min(e, 31);
+    uint32_t vis = (lo <= hi) ? ((0xffffffffu << lo) & (0xffffffffu >> (31 - hi))) : 0u;
+    if (pre > 0) vis |= (pre >= 32) ? 0xffffffffu : ((1u << pre) - 1u);
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (!(vis & (1u << i))) y[i] = __float_as_uint(-INFINITY);
 }
-// Publishes this warp's TMEM stores to the MMA thread: every lane waits for its own stores first.
-__device__ __forceinline__ void warp_arrive_after_tmem_st(uint32_t bar) {
-    ptx::tmem_wait_st();
-    ptx::tc_fence_before_sync();
-    warp_arrive(bar);
+__device__ __forceinline__ void mask_chunk32_cmp(uint32_t* y, int a, int e) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+        if (i < a || i > e) y[i] = __float_as_uint(-INFINITY);
 }
 
 // exp2 of 32 shifted scores -> 16 packed bf16 pairs; accumulates the fp32 row sum in four packed lanes.
@@ -66,6 +75,21 @@ __device__ __forceinline__ void exp_chunk(const uint32_t* y, float cs, float neg
 }
 
 // ------------------------------------------------------------------------------------------------ host side
+// The opt-in shared-memory size is a per-device attribute of each kernel: set by the first call on a device.
+// `done` is the calling launcher's own flag array (one per kernel instance).  Host threads may race on the first
+// call: the flags are atomic and setting the attribute twice is harmless.
+using SmemAttrFlags = std::atomic<bool>[64];
+template <typename Kernel>
+inline bool set_smem_attr_once(SmemAttrFlags& done, Kernel kernel, int bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const bool tracked = dev >= 0 && dev < 64;
+    if (tracked && done[dev].load(std::memory_order_acquire)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (tracked) done[dev].store(true, std::memory_order_release);
+    return true;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -84,17 +108,32 @@ inline EncodeTiledFn encode_fn() {
 
 // bf16 tensor [B, H, S, D] with element strides st (batch, head, row): box = box_cols columns x box_rows rows,
 // 128-byte swizzle (the layout tcgen05.mma reads directly).
-inline bool make_map(CUtensorMap* map, const void* ptr, int B, int H, int S, int D, const long long st[3], int box_rows,
-                     int box_cols = 64) {
+struct MapKey {
+    const void* ptr;
+    int B, H, S, D;
+    long long st[3];
+    int box_rows, box_cols;
+};
+inline bool encode_map(CUtensorMap* map, const MapKey& k) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)S, (cuuint64_t)H, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)st[2] * 2, (cuuint64_t)st[1] * 2, (cuuint64_t)st[0] * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1u, 1u};
+    const cuuint64_t dims[4] = {(cuuint64_t)k.D, (cuuint64_t)k.S, (cuuint64_t)k.H, (cuuint64_t)k.B};
+    const cuuint64_t strides[3] = {(cuuint64_t)k.st[2] * 2, (cuuint64_t)k.st[1] * 2, (cuuint64_t)k.st[0] * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)k.box_cols, (cuuint32_t)k.box_rows, 1u, 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k.ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Encoded maps are cached by key (attn_api.cu; emptied by attn_clear_cache()).
+bool cached_map(CUtensorMap* out, const MapKey& key);
+void clear_map_cache();
+long long map_cache_hits();
+
+inline bool make_map(CUtensorMap* map, const void* ptr, int B, int H, int S, int D, const long long st[3], int box_rows,
+                     int box_cols = 64) {
+    const MapKey key = {ptr, B, H, S, D, {st[0], st[1], st[2]}, box_rows, box_cols};
+    return cached_map(map, key);
 }
 
 }  // namespace tc

@@ -125,44 +125,13 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int pair) {
     return it;
 }
 
-template <bool kCluster>
-__device__ __forceinline__ bool bounded_wait_t(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    auto attempt = [&]() { return kCluster ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity); };
-    if (attempt()) return true;
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    volatile int* abort_flag = &bars->abort_flag;
-    while (true) {
-        if (attempt()) return true;
-        if ((++spins & 0x3Fu) == 0) {
-            if (*abort_flag) return false;
-            const uint64_t now = ptx::globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (status_word) atomicExch(status_word, (int)ATTN_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    return bounded_wait_t<false>(bar, parity, bars, status_word);
+    return bounded_wait_on<false>(bar, parity, &bars->abort_flag, status_word);
 }
 // For barriers that the other CTA of the pair arrives on.
 __device__ __forceinline__ bool bounded_wait_cluster(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    return bounded_wait_t<true>(bar, parity, bars, status_word);
+    return bounded_wait_on<true>(bar, parity, &bars->abort_flag, status_word);
 }
-
-#ifdef ATTN_DEBUG_TRACE
-// Debug build only: CTA 0 records clock() stamps of its first 24 key tiles into the int32 array behind
-// status_word, [event * 32 + n]: 0 S seen, 1 S in registers, 2 maxima exchanged, 3 P published, 4 MMA thread saw P
-// of both CTAs, 5 P V issued, 6 next Q K^T issued, 7 MMA thread has the K/V slots.
-#define TRACE(ev, n) do { if (blockIdx.x == 0 && (n) < 24 && p.status_word) p.status_word[(ev) * 32 + (n)] = (int)clock(); } while (0)
-#else
-#define TRACE(ev, n)
-#endif
 
 // Waits for the next work item published by the leader's scheduler thread and releases the slot.
 // Returns false when the grid has no unstarted cluster left (or the wait was abandoned).
@@ -190,16 +159,10 @@ __device__ __forceinline__ void scheduler_role(Barriers* bars, int32_t* status_w
         if (rank == 0) {
             if (!bounded_wait_cluster(ptx::smem_u32(&bars->item_ready), ready_phase, bars, status_word)) return;
             ready_phase ^= 1u;
-            const uint32_t bar = ptx::smem_u32(&bars->clc);
-            ptx::mbar_arrive_expect_tx(bar, 16);
-            ptx::clc_try_cancel(ptx::smem_u32(&bars->clc_response[0]), bar);
-            if (!bounded_wait(bar, clc_phase, bars, status_word)) return;
-            clc_phase ^= 1u;
-            const uint64_t lo = *reinterpret_cast<volatile uint64_t*>(&bars->clc_response[0]);
-            const uint64_t hi = *reinterpret_cast<volatile uint64_t*>(&bars->clc_response[1]);
+            bool handed;
             uint32_t x;
-            const uint32_t got = ptx::clc_query(lo, hi, x) ? 1u : 0u;
-            ptx::fence_proxy_async_smem();   // these generic-proxy reads come before the next try_cancel's async write
+            if (!clc_fetch(ptx::smem_u32(&bars->clc), bars->clc_response, clc_phase, &bars->abort_flag, status_word, handed, x)) return;
+            const uint32_t got = handed ? 1u : 0u;
             // Publish {got, index} in both CTAs, then signal each CTA's item_full.
 #pragma unroll
             for (uint32_t r = 0; r < 2; ++r) {
@@ -366,9 +329,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
             for (int j = J0; j < J1; ++j, ++g) {
                 const int buf = (int)(g % NS);
                 const uint32_t ph = (g / NS) & 1u;
-                TRACE(7, j - J0);
                 if (j + NS - 1 < J1 && !qk_step(j + NS - 1, g + NS - 1, J1)) return;
-                TRACE(6, j - J0);
                 int vslot;
                 if (!next_slot(vslot)) return;
                 // Before the first P V of an item overwrites O: both epilogues of the previous item must have read it.
@@ -376,7 +337,6 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
                     if (!bounded_wait(ptx::smem_u32(&bars->o_free), (uint32_t)((q_uses - 1) & 1), bars, p.status_word)) return;
                 }
                 if (!bounded_wait(bar_p_full + buf * 8, ph, bars, p.status_word)) return;
-                TRACE(4, j - J0);
                 ptx::tc_fence_after_sync();
                 if constexpr (P_HI_LO) {
                     // P = P_hi + P_lo, two bf16 tiles 32 columns apart inside each group's S columns.
@@ -387,7 +347,6 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
                 }
                 ptx::tc_commit_pair(bar_pv_done + buf * 8);
                 if (j == J1 - 1) ptx::tc_commit_pair(ptx::smem_u32(&bars->o_done));
-                TRACE(5, j - J0);
                 ptx::tc_commit_pair(bar_empty + vslot * 8);
             }
             ++q_uses;
@@ -474,7 +433,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             const float rowoff = (float)(ip - kv0 - col0);
             const uint32_t ts = tm + buf * kBN + col0;        // this thread's lane, this group's S / P columns
             if (!bounded_wait(ptx::smem_u32(&bars->s_full[buf]), ph, bars, p.status_word)) return;
-            if (threadIdx.x == 0) TRACE(0, n);
             ptx::tc_fence_after_sync();
 
             // y: scores in log2 units (SCORE plain: raw, scaled inside the max / exp steps), masked to -inf.
@@ -484,16 +442,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             ptx::tmem_ld_32x32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&y[32]));
             ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[0]));
             ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[32]));
-            if (threadIdx.x == 0) TRACE(1, n);
 #pragma unroll
             for (int c = 0; c < kWgCols / 32; ++c) {
                 // Score (Appendix A.1)
                 if constexpr (SCORE != kScorePlain) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
-                if (!full_tile) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c * 32 + i < mask_a || c * 32 + i > mask_e) y[c * 32 + i] = __float_as_uint(-INFINITY);
-                }
+                if (!full_tile) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);   // (the bit-test form cost this kernel 2 %)
                 if (!SIGMOID && !RELU && !fixed_max) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -545,7 +498,6 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 if constexpr (SCORE == kScorePlain) mt *= cs;
                 float mt_other;
                 if (!exchange(mt, mt_other)) return;
-                if (threadIdx.x == 0) TRACE(2, n);
                 const float m_new = fmaxf(m_used, fmaxf(mt, mt_other));   // identical in both groups
                 if (n == 0) {
                     m_used = m_new;
@@ -592,14 +544,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                     ptx::unpack2(ptx::add2(sume[0], sume[1]), s0, s1);
                     l_exact += s0 + s1;
                 }
-                if (threadIdx.x == 0) TRACE(8, n);
             }
             // Publish this warp's P (and any rescaled O) to the MMA thread of the leader CTA.
             ptx::tmem_wait_st();
-            if (threadIdx.x == 0) TRACE(9, n);
             ptx::tc_fence_before_sync();
             warp_arrive_on_leader(p_full_on_leader + buf * 8);
-            if (threadIdx.x == 0) TRACE(3, n);
         }
 
         // Epilogue: O / l (softmax), O * out_scale (sigmoid) or O * out_scale * ln 2 (ReLU: P was kept in log2 units);
@@ -741,6 +690,8 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
             if (lane == 0 && rank == 0) mma_role<D, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
             if (lane == 0) scheduler_role(bars, p.status_word, rank);
+        } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
+            check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
         __syncwarp();
     }
@@ -761,14 +712,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     using C = Cfg<D>;
     auto kernel = attn_fwd_pair_kernel<D, SCORE, NORM>;
     // The opt-in shared-memory size is a per-device function attribute: set it once per device.
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    static SmemAttrFlags attr_set;
+    if (!set_smem_attr_once(attr_set, kernel, C::kSmemBytes)) return ATTN_ERR_CUDA;
     CUtensorMap mq, mk, mv;
     if (!make_map(&mq, p.q, p.B, p.Hq, p.Sq, D, p.qs, 128) || !make_map(&mk, p.k, p.B, p.Hkv, p.Sk, D, p.ks, 64) ||
         !make_map(&mv, p.v, p.B, p.Hkv, p.Sk, D, p.vs, 128))

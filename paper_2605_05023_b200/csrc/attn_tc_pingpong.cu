@@ -93,15 +93,7 @@ struct Barriers {
     int item_msg[kItemWords + 1];   // {a work item was handed over, the decoded Item}, written by the scheduler thread
     uint32_t tmem_base;
     int abort_flag;
-#ifdef ATTN_DEBUG_WHERE
-    int dbg[16];             // debug build: last progress mark of every warp
-#endif
 };
-#ifdef ATTN_DEBUG_WHERE
-#define DBG_MARK(v) do { if ((threadIdx.x & 31) == 0) ((volatile int*)bars->dbg)[threadIdx.x >> 5] = (int)(v); } while (0)
-#else
-#define DBG_MARK(v)
-#endif
 static_assert(sizeof(Barriers) <= 1024, "barrier block");
 
 struct TileRange {
@@ -175,47 +167,7 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
 }
 
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    volatile int* abort_flag = &bars->abort_flag;
-    while (true) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3Fu) == 0) {
-#ifdef ATTN_DEBUG_WHERE
-            if (*abort_flag) {
-                if (status_word && (int)blockIdx.x == *(volatile int*)(status_word + 5)) {
-                    status_word[16 + (threadIdx.x >> 5) * 2] = (int)(bar - ptx::smem_u32(bars));
-                    status_word[17 + (threadIdx.x >> 5) * 2] = (int)parity + 100;
-                }
-                return false;
-            }
-#else
-            if (*abort_flag) return false;
-#endif
-            const uint64_t now = ptx::globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (status_word) atomicExch(status_word, (int)ATTN_ERR_TIMEOUT);
-#ifdef ATTN_DEBUG_WHERE
-                // Debug build only: the first wait that gave up records its barrier (byte offset in the barrier
-                // block), parity, thread and CTA in status words 2..5; the other warps of that CTA then record
-                // what they were waiting for in words 16 + 2 * warp (offset) and 17 + 2 * warp (parity + 100).
-                if (status_word && atomicCAS(status_word + 1, 0, 1) == 0) {
-                    status_word[2] = (int)(bar - ptx::smem_u32(bars));
-                    status_word[3] = (int)parity;
-                    status_word[4] = (int)threadIdx.x;
-                    status_word[5] = (int)blockIdx.x;
-                    for (int w = 0; w < 12; ++w) status_word[40 + w] = ((volatile int*)bars->dbg)[w];
-                    __threadfence();
-                }
-#endif
-                return false;
-            }
-        }
-    }
+    return bounded_wait_on<false>(bar, parity, &bars->abort_flag, status_word);
 }
 
 // Waits for the next work item published by the scheduler thread, copies it and (kRelease) releases it.  The
@@ -240,13 +192,9 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
 // scheduler: one thread
 // ------------------------------------------------------------------------------------------------
 // Fetches work items one ahead and decodes them for everybody: the first item is this CTA's own index, the
-// following ones are CTAs of the grid that have not started, taken over with cluster launch control.  Only this
-// thread touches the 16 response bytes that the hardware scheduler writes through the async proxy: it decodes
-// them and publishes {handed over, decoded item} with ordinary stores for the other roles, so that no role
-// spends time on index arithmetic and mask intervals.  Its reads of the response are ordered before the next
-// request's write by a proxy fence.  (With every role reading the response itself and no such fence, a late
-// reader now and then saw the bytes of the following response: one warp left the work loop early and its query
-// tile's barriers were never completed.)
+// following ones are CTAs of the grid that have not started, taken over with cluster launch control (clc_fetch:
+// only this thread touches the hardware scheduler's response).  It publishes {handed over, decoded item} with
+// ordinary stores for the other roles, so that no role spends time on index arithmetic and mask intervals.
 template <int NQ>
 __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* bars) {
     int32_t* status_word = p.status_word;
@@ -269,16 +217,9 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
         // every role has copied the published item: fetch the next one
         if (!bounded_wait(ptx::smem_u32(&bars->item_empty), empty_phase, bars, status_word)) return;
         empty_phase ^= 1u;
-        const uint32_t bar = ptx::smem_u32(&bars->clc);
-        ptx::mbar_arrive_expect_tx(bar, 16);
-        ptx::clc_try_cancel(ptx::smem_u32(&bars->item_response[0]), bar);
-        if (!bounded_wait(bar, clc_phase, bars, status_word)) return;
-        clc_phase ^= 1u;
-        const uint64_t lo = *reinterpret_cast<volatile uint64_t*>(&bars->item_response[0]);
-        const uint64_t hi = *reinterpret_cast<volatile uint64_t*>(&bars->item_response[1]);
+        bool got;
         uint32_t x;
-        const bool got = ptx::clc_query(lo, hi, x);
-        ptx::fence_proxy_async_smem();
+        if (!clc_fetch(ptx::smem_u32(&bars->clc), bars->item_response, clc_phase, &bars->abort_flag, status_word, got, x)) return;
         publish(got, (int)x);
         if (!got) return;                           // no item left: stop asking
     }
@@ -613,19 +554,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
                     }
                     if (kMasked) {
-                        if constexpr (SIGMOID || RELU) {
-    #pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (c * 32 + i < mask_a || c * 32 + i > mask_e) y[c * 32 + i] = __float_as_uint(-INFINITY);
-                        } else {
-                            // Visible columns of this row inside the chunk as a 32-bit word: one bit test per element
-                            // (two compares per element made partial tiles cost half as much again as full ones).
-                            const int lo = max(mask_a - c * 32, 0), hi = min(mask_e - c * 32, 31);
-                            const uint32_t vis = (lo <= hi) ? ((0xffffffffu << lo) & (0xffffffffu >> (31 - hi))) : 0u;
-    #pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (!(vis & (1u << i))) y[c * 32 + i] = __float_as_uint(-INFINITY);
-                        }
+                        // One bit test per element (two compares per element made partial tiles cost half as much
+                        // again as full ones); the sigmoid and ReLU instances are faster with the compare form.
+                        if constexpr (SIGMOID || RELU) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
+                        else mask_chunk32_bits(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
                     }
                     if constexpr (!SIGMOID && !RELU) {
     #pragma unroll
@@ -818,9 +750,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         ptx::mbar_init(ptx::smem_u32(&bars->item_full), 1);
         ptx::mbar_init(ptx::smem_u32(&bars->item_empty), C::kItemConsumers);
         bars->abort_flag = 0;
-#ifdef ATTN_DEBUG_WHERE
-        for (int w = 0; w < 16; ++w) bars->dbg[w] = 0;
-#endif
         ptx::fence_mbar_init();
         ptx::fence_proxy_async_smem();
     }
@@ -837,7 +766,6 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp < NQ * 4) {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         softmax_role<D, NQ, SCORE, NORM>(p, bars, tmem, warp >> 2);
-        DBG_MARK(9000000);
     } else {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         if (warp == C::kProducerWarp) {
@@ -846,6 +774,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
             if (lane == 0) mma_role<D, NQ, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
             if (lane == 0) scheduler_role<NQ>(p, bars);
+        } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
+            check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
         __syncwarp();
     }
@@ -866,14 +796,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     using C = Cfg<D, NQ>;
     auto kernel = attn_fwd_tc_kernel<D, NQ, SCORE, NORM>;
     // The opt-in shared-memory size is a per-device function attribute: set it once per device.
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    static SmemAttrFlags attr_set;
+    if (!set_smem_attr_once(attr_set, kernel, C::kSmemBytes)) return ATTN_ERR_CUDA;
     CUtensorMap mq, mk, mv;
     if (!make_map(&mq, p.q, p.B, p.Hq, p.Sq, D, p.qs, 128) || !make_map(&mk, p.k, p.B, p.Hkv, p.Sk, D, p.ks, 128) ||
         !make_map(&mv, p.v, p.B, p.Hkv, p.Sk, D, p.vs, 128))
@@ -923,7 +847,7 @@ int launch_attn_fwd_bf16(const AttnParams& p, cudaStream_t stream, int* launches
     static const bool force_split = []() { const char* e = getenv("B200ATTN_FORCE_SPLIT"); return e && e[0] == '1'; }();
     static const bool force_pair = []() { const char* e = getenv("B200ATTN_FORCE_PAIR"); return e && e[0] == '1'; }();
     int rc;
-    if (force_split || p.global_len > 0) {      // two key intervals per row: only the one-tile kernel walks them
+    if (force_split || (p.mask_flags & kMaskGlobal)) {      // two key intervals per row: only the one-tile kernel walks them
         rc = launch_attn_fwd_bf16_split(p, stream);
     } else if (p.D == 256 || (force_pair && p.D == 128)) {
         rc = launch_attn_fwd_bf16_pair(p, stream);

@@ -136,24 +136,7 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
 }
 
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    volatile int* abort_flag = &bars->abort_flag;
-    while (true) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3Fu) == 0) {
-            if (*abort_flag) return false;
-            const uint64_t now = ptx::globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (status_word) atomicExch(status_word, (int)ATTN_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
+    return bounded_wait_on<false>(bar, parity, &bars->abort_flag, status_word);
 }
 
 // Waits for the next work item published by the scheduler thread and releases it.
@@ -170,26 +153,16 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
 // ------------------------------------------------------------------------------------------------
 // scheduler: one thread
 // ------------------------------------------------------------------------------------------------
-// Only this thread touches the 16 response bytes that the hardware scheduler writes through the async proxy: it
-// decodes them and publishes {handed over, index} with ordinary stores for the other roles.  Its reads of the
-// response are ordered before the next request's write by a proxy fence.  (With every role reading the response
-// itself and no such fence, a late reader now and then saw the bytes of the following response: one warp left
-// the work loop early and its query tile's barriers were never completed.)
+// Only this thread touches the hardware scheduler's response (clc_fetch); it publishes {handed over, index} with
+// ordinary stores for the other roles.
 __device__ __forceinline__ void scheduler_role(Barriers* bars, int32_t* status_word) {
     uint32_t clc_phase = 0, empty_phase = 1;        // the first wait on item_empty passes at once
     while (true) {
         if (!bounded_wait(ptx::smem_u32(&bars->item_empty), empty_phase, bars, status_word)) return;
         empty_phase ^= 1u;
-        const uint32_t bar = ptx::smem_u32(&bars->clc);
-        ptx::mbar_arrive_expect_tx(bar, 16);
-        ptx::clc_try_cancel(ptx::smem_u32(&bars->item_response[0]), bar);
-        if (!bounded_wait(bar, clc_phase, bars, status_word)) return;
-        clc_phase ^= 1u;
-        const uint64_t lo = *reinterpret_cast<volatile uint64_t*>(&bars->item_response[0]);
-        const uint64_t hi = *reinterpret_cast<volatile uint64_t*>(&bars->item_response[1]);
+        bool got;
         uint32_t x;
-        const bool got = ptx::clc_query(lo, hi, x);
-        ptx::fence_proxy_async_smem();
+        if (!clc_fetch(ptx::smem_u32(&bars->clc), bars->item_response, clc_phase, &bars->abort_flag, status_word, got, x)) return;
         *reinterpret_cast<volatile uint32_t*>(&bars->item_value[0]) = got ? 1u : 0u;
         *reinterpret_cast<volatile uint32_t*>(&bars->item_value[1]) = x;
         ptx::mbar_arrive(ptx::smem_u32(&bars->item_full));
@@ -473,17 +446,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             for (int c = 0; c < kWgCols / 32; ++c) {
                 // Score (Appendix A.1)
                 if constexpr (SCORE != kScorePlain) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
-                if (!full_tile) {
-                    // Visible columns of this row inside the chunk as a 32-bit word (the row's interval and, for global
-                    // tokens, the columns below mask_p): one bit test per element.
-                    const int lo = max(mask_a - c * 32, 0), hi = min(mask_e - c * 32, 31);
-                    const int pre = min(max(mask_p - c * 32, 0), 32);
-                    const uint32_t vis = ((lo <= hi) ? ((0xffffffffu << lo) & (0xffffffffu >> (31 - hi))) : 0u) |
-                                         (pre >= 32 ? 0xffffffffu : ((1u << pre) - 1u));
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (!(vis & (1u << i))) y[c * 32 + i] = __float_as_uint(-INFINITY);
-                }
+                // the row's interval and, for global tokens, the columns below mask_p
+                if (!full_tile) mask_chunk32_bits(&y[c * 32], mask_a - c * 32, mask_e - c * 32, mask_p - c * 32);
                 if constexpr (!SIGMOID && !RELU) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -707,6 +671,8 @@ attn_fwd_split_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             if (lane == 0) mma_role<D, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
             if (lane == 0) scheduler_role(bars, p.status_word);
+        } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
+            check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
         __syncwarp();
     }
@@ -727,14 +693,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     using C = Cfg<D>;
     auto kernel = attn_fwd_split_kernel<D, SCORE, NORM>;
     // The opt-in shared-memory size is a per-device function attribute: set it once per device.
-    static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return ATTN_ERR_CUDA;
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-            return ATTN_ERR_CUDA;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
+    static SmemAttrFlags attr_set;
+    if (!set_smem_attr_once(attr_set, kernel, C::kSmemBytes)) return ATTN_ERR_CUDA;
     CUtensorMap mq, mk, mv;
     if (!make_map(&mq, p.q, p.B, p.Hq, p.Sq, D, p.qs, 128) || !make_map(&mk, p.k, p.B, p.Hkv, p.Sk, D, p.ks, 128) ||
         !make_map(&mv, p.v, p.B, p.Hkv, p.Sk, D, p.vs, D == 256 ? 64 : 128))

@@ -30,12 +30,9 @@ bool host_layout(int M, int N, int K, HostLayout* L) {
     return true;
 }
 
-}  // namespace
-
-extern "C" {
-
-int gemm_rowsum(const void* a, const void* b, void* c, float* rowsum, int M, int N, int K,
-                const gemm_rowsum_desc* desc, void* stream) {
+// Every argument check of gemm_rowsum, made before any CUDA call; fills the launch parameters.
+int check_and_fill(const void* a, const void* b, void* c, float* rowsum, int M, int N, int K,
+                   const gemm_rowsum_desc* desc, b200attn::GemmRowsumParams* out) {
     if (!a || !b || !rowsum) return ATTN_ERR_NULL;
     if (M <= 0 || N <= 0 || K <= 0) return ATTN_ERR_SHAPE;
     if (desc && (desc->struct_size != sizeof(gemm_rowsum_desc) || desc->reserved != 0)) return ATTN_ERR_DESC;
@@ -52,9 +49,19 @@ int gemm_rowsum(const void* a, const void* b, void* c, float* rowsum, int M, int
     if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c)) & 15u) return ATTN_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(rowsum) & 3u) return ATTN_ERR_ALIGN;
     if ((p.lda | p.ldb | p.ldc) & 7 || (N & 7)) return ATTN_ERR_ALIGN;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(rowsum, 0, (size_t)M * sizeof(float), st) != cudaSuccess) return ATTN_ERR_CUDA;
-    const int rc = b200attn::launch_gemm_rowsum_bf16(p, st);
+    *out = p;
+    return ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gemm_rowsum(const void* a, const void* b, void* c, float* rowsum, int M, int N, int K,
+                const gemm_rowsum_desc* desc, void* stream) {
+    b200attn::GemmRowsumParams p;
+    if (const int rc = check_and_fill(a, b, c, rowsum, M, N, K, desc, &p)) return rc;
+    const int rc = b200attn::launch_gemm_rowsum_bf16(p, reinterpret_cast<cudaStream_t>(stream));
     if (rc == ATTN_OK) g_gemm_launches.fetch_add(1, std::memory_order_relaxed);
     return rc;
 }
@@ -75,11 +82,17 @@ int gemm_rowsum_host(const void* a_host, const void* b_host, void* c_host, float
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return ATTN_ERR_ALIGN;
     char* ws = static_cast<char*>(workspace);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // Every argument check runs before the first copy is enqueued: on an argument error nothing reaches the stream.
+    b200attn::GemmRowsumParams p;
+    if (const int rc = check_and_fill(ws + L.a, ws + L.b, c_host ? ws + L.c : nullptr, reinterpret_cast<float*>(ws + L.r), M, N, K,
+                                      desc, &p))
+        return rc;
     if (cudaMemcpyAsync(ws + L.a, a_host, L.ab, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaMemcpyAsync(ws + L.b, b_host, L.bb, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return ATTN_ERR_CUDA;
-    const int rc = gemm_rowsum(ws + L.a, ws + L.b, c_host ? ws + L.c : nullptr, reinterpret_cast<float*>(ws + L.r), M, N, K, desc, stream);
+    const int rc = b200attn::launch_gemm_rowsum_bf16(p, st);
     if (rc != ATTN_OK) return rc;
+    g_gemm_launches.fetch_add(1, std::memory_order_relaxed);
     if (c_host && cudaMemcpyAsync(c_host, ws + L.c, L.cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ATTN_ERR_CUDA;
     if (cudaMemcpyAsync(rowsum_host, ws + L.r, L.rb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ATTN_ERR_CUDA;
     return ATTN_OK;

@@ -80,24 +80,7 @@ struct Barriers {
 static_assert(sizeof(Barriers) <= kBarBytes, "barrier block");
 
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    uint64_t t0 = 0;
-    uint32_t spins = 0;
-    volatile int* abort_flag = &bars->abort_flag;
-    while (true) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 0x3Fu) == 0) {
-            if (*abort_flag) return false;
-            const uint64_t now = ptx::globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (status_word) atomicExch(status_word, (int)ATTN_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
+    return bounded_wait_on<false>(bar, parity, &bars->abort_flag, status_word);
 }
 
 // Tile t of the pair's round-robin sequence: first n_wide tiles of 256 columns, then narrow tiles of 128 columns
@@ -349,21 +332,21 @@ namespace {
 // (a GPC with an odd number of free SMs leaves one of them without a partner).
 template <int kAccs>
 int prepare(int dev, cudaLaunchConfig_t& cfg, int& max_pairs_out) {
-    static bool attr_set[64] = {};
-    static int max_pairs[64] = {};
+    static std::atomic<bool> attr_set[64];      // host threads may race on the first call: both compute the same values
+    static std::atomic<int> max_pairs[64];
     auto kernel = gemm_rowsum_pair_kernel<kAccs>;
     cfg.dynamicSmemBytes = Cfg<kAccs>::kSmemBytes;
-    if (!attr_set[dev]) {
+    if (!attr_set[dev].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<kAccs>::kSmemBytes) != cudaSuccess)
             return ATTN_ERR_CUDA;
         int sms = 0, n = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) return ATTN_ERR_CUDA;
         cfg.gridDim = dim3((unsigned)(sms / 2 * 2), 1, 1);
         if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) return ATTN_ERR_CUDA;
-        max_pairs[dev] = n < sms / 2 ? n : sms / 2;
-        attr_set[dev] = true;
+        max_pairs[dev].store(n < sms / 2 ? n : sms / 2, std::memory_order_relaxed);
+        attr_set[dev].store(true, std::memory_order_release);
     }
-    max_pairs_out = max_pairs[dev];
+    max_pairs_out = max_pairs[dev].load(std::memory_order_relaxed);
     return ATTN_OK;
 }
 
@@ -405,6 +388,7 @@ int launch_gemm_rowsum_bf16(GemmRowsumParams p, cudaStream_t stream) {
         p.n_wide = p.n_tiles = (int)big_tiles;
         const long long pairs = big_tiles < P2 ? big_tiles : P2;
         cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+        if (cudaMemsetAsync(p.rowsum, 0, (size_t)p.M * sizeof(float), stream) != cudaSuccess) return ATTN_ERR_CUDA;
         return cudaLaunchKernelEx(&cfg, gemm_rowsum_pair_kernel<2>, ma, mb, p) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
     }
 
@@ -423,6 +407,8 @@ int launch_gemm_rowsum_bf16(GemmRowsumParams p, cudaStream_t stream) {
     p.n_tiles = (int)(split ? tiles + n_split : tiles);
     const long long pairs = p.n_tiles < P1 ? p.n_tiles : P1;
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    // The row sums are cleared on the caller's stream only now, after everything that can fail on the host.
+    if (cudaMemsetAsync(p.rowsum, 0, (size_t)p.M * sizeof(float), stream) != cudaSuccess) return ATTN_ERR_CUDA;
     return cudaLaunchKernelEx(&cfg, gemm_rowsum_pair_kernel<1>, ma, mb, p) == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 

@@ -12,7 +12,7 @@ import torch
 
 import paper_2605_05023_b200 as pk
 from paper_2605_05023_b200 import binding
-from paper_2605_05023_b200.flops import row_visibility, unmasked_flops, visible_pairs
+from workload_flops import row_visibility, unmasked_flops, visible_pairs
 from synth_inputs import Workload, benchmark_workloads
 
 from helpers import visible_matrix
@@ -29,7 +29,8 @@ def declared_functions(header="attn.h", prefix="attn_"):
 def test_library_exports_every_declared_symbol():
     names = declared_functions()
     assert {"attn_fwd", "attn_fwd_host", "attn_host_workspace_bytes", "attn_status_string",
-            "attn_version", "attn_launch_count"} <= set(names)
+            "attn_version", "attn_launch_count", "attn_clear_cache", "attn_cache_hits",
+            "attn_selftest_timeout"} <= set(names)
     lib = ctypes.CDLL(binding.LIB_PATH)
     for n in names:
         assert hasattr(lib, n), n
@@ -100,6 +101,59 @@ def test_host_entry_point_validation():
     d2 = good_desc(q_strides=(ctypes.c_int64 * 3)(8, 8, 8))
     rc = lib.attn_fwd_host(FAKE, FAKE, FAKE, FAKE, None, 1, 2, 2, 128, 128, 128, ctypes.byref(d2), FAKE, 1 << 30, None)
     assert rc == 5
+
+
+def test_host_entry_point_checks_every_argument_before_the_first_copy():
+    """An argument error of the staged entry points must leave nothing on the stream: with a workspace that is
+    large enough, the answer is the argument's own status (a copy would have been a CUDA call: status 6 here)."""
+    lib = binding._lib
+    for kw, sizes, status in [
+        (dict(), dict(D=96), 3),                                   # unsupported head dimension
+        (dict(normalizer=7), dict(), 5),
+        (dict(dtype=9), dict(), 5),
+        (dict(mask_flags=binding.ATTN_MASK_DOCUMENT), dict(), 5),  # document mask without offsets
+        (dict(), dict(Hq=3, Hkv=2), 2),
+    ]:
+        d = good_desc(**kw)
+        a = dict(B=1, Hq=2, Hkv=2, Sq=128, Sk=128, D=128)
+        a.update(sizes)
+        before = pk.launch_count()
+        rc = lib.attn_fwd_host(FAKE, FAKE, FAKE, FAKE, None, a["B"], a["Hq"], a["Hkv"], a["Sq"], a["Sk"], a["D"],
+                               ctypes.byref(d), FAKE * 16, 1 << 30, None)
+        assert rc == status, (kw, sizes, rc)
+        assert pk.launch_count() == before
+    # the GEMM twin: N not a multiple of 8 is an alignment error, found before the copies
+    rc = lib.gemm_rowsum_host(FAKE, FAKE, FAKE, FAKE, 128, 100, 64, None, FAKE * 16, 1 << 30, None)
+    assert rc == 4
+
+
+def test_cache_and_selftest_entry_points_validate_on_the_host():
+    assert pk.clear_cache() == 0                                   # host memory only: works without a GPU
+    assert pk.cache_hits() >= 0
+    lib = binding._lib
+    assert lib.attn_selftest_timeout(None, 1000, None, None) == 1
+    assert lib.attn_selftest_timeout(FAKE + 2, 1000, None, None) == 4
+    assert lib.attn_selftest_timeout(FAKE, 0, None, None) == 5
+    assert lib.attn_selftest_timeout(FAKE, 10**9, None, None) == 5  # beyond 0.1 s
+
+
+def test_concurrent_host_threads_get_the_same_answers():
+    """Argument checks and the tensor-map cache bookkeeping from eight host threads at once."""
+    import threading
+    out = []
+
+    def work():
+        d = good_desc()
+        codes = [pk.raw_attn_fwd(FAKE, FAKE, FAKE, FAKE, FAKE, 1, 6, 4, 128, 128, 128, d, None) for _ in range(200)]
+        codes += [pk.clear_cache() for _ in range(50)]
+        out.append(set(codes))
+
+    threads = [threading.Thread(target=work) for _ in range(8)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert out == [{2, 0}] * 8
 
 
 def test_cpu_tensors_are_refused():

@@ -30,13 +30,32 @@ def gpu_run(w, q, k, v, poison=True):
     return o, lse
 
 
+def relu_row_bounds(w, v, o_ref, p_ref):
+    """Per-element error bound of the ReLU normaliser, scaled by what each ROW holds (a row of small outputs
+    gets a small bound).  O_id = sum_j P_ij V_jd with P rounded to bf16 before the product (relative error up
+    to 2^-9 per weight, independent signs: standard deviation 2^-9 / sqrt(3) * sqrt(sum_j (P_ij V_jd)^2), taken
+    at six sigma = 2^-7) and O rounded once to the output type (2^-9 relative for bf16).  fp32 inputs: every
+    step is fp32, 1e-5 of the same two row quantities."""
+    B, Hq, Sq, D = o_ref.shape
+    g = Hq // w.Hkv
+    v2 = (v.double().numpy() ** 2).repeat(g, axis=1)                      # [B, Hq, Sk, D]
+    spread = np.sqrt(np.einsum("bhij,bhjd->bhid", p_ref ** 2, v2))
+    if w.dtype == "bf16":
+        out_round = 2.0 ** -9 if w.o_dtype == "bf16" else 2.0 ** -23
+        return 2.0 ** -7 * spread + out_round * np.abs(o_ref) + 1e-30
+    return 1e-5 * (spread + np.abs(o_ref)) + 1e-30
+
+
 def check(w, rows=None):
     q, k, v = make_qkv(w)
     o, lse = gpu_run(w, q, k, v)
     tol_o, tol_l = TOL[w.dtype]
     o_np = o.double().cpu().numpy()
     if rows is None:
-        o_ref, lse_ref = oracle_run(w, q, k, v)
+        if w.normalizer == "relu":
+            o_ref, lse_ref, p_ref = oracle_run(w, q, k, v, want_p=True)
+        else:
+            o_ref, lse_ref = oracle_run(w, q, k, v)
         l_np = None if lse is None else lse.double().cpu().numpy()
     else:
         o_ref, lse_ref = oracle_run(w, q, k, v, rows=rows)
@@ -45,8 +64,13 @@ def check(w, rows=None):
     assert not np.isnan(o_np).any(), "unwritten or NaN output rows"
     if w.normalizer == "relu":
         # out_scale * max(s, 0) has no row normalisation: the output scale is set by out_scale and the sequence
-        # length, so the bound is relative to the largest output (bf16 P and bf16 O round at up to 2^-8 relative).
+        # length, so the bound is relative to the largest output (bf16 P and bf16 O round at up to 2^-8 relative) ...
         tol_o = tol_o * max(float(np.abs(o_ref).max()), 1e-30) * (0.5 if w.dtype == "bf16" else 1.0)
+        # ... and, so that a row of small outputs cannot hide a large relative error, every element is also held to
+        # a bound scaled by its own row.
+        if rows is None:
+            ratio = np.abs(o_np - o_ref) / relu_row_bounds(w, v, o_ref, p_ref)
+            assert ratio.max() <= 1.0, f"{w.name}: per-row ReLU bound exceeded {ratio.max():.2f} times"
     err_o = np.abs(o_np - o_ref).max()
     assert err_o <= tol_o, f"{w.name}: max|dO| = {err_o:.3e} > {tol_o}"
     if l_np is not None:
@@ -80,6 +104,16 @@ FP32_CASES = [
              cu_seqlens=(0, 70, 71, 130, 200), global_len=70),
     Workload("f_global_causal_sq_lt_sk", 1, 1, 1, 90, 150, 64, dtype="fp32", o_dtype="fp32", seed=63, causal=True,
              window_left=10, window_right=0, global_len=5),
+    # more query rows than keys (i' = i + Sk - Sq < 0 for the first rows) under masks other than plain causal
+    Workload("f_sq_gt_sk_window", 1, 2, 1, 100, 40, 32, dtype="fp32", o_dtype="fp32", seed=76, window_left=7, window_right=9),
+    Workload("f_sq_gt_sk_prefix_window", 1, 1, 1, 90, 50, 64, dtype="fp32", o_dtype="fp32", seed=77, causal=True,
+             prefix_len=20, window_left=12, window_right=0),
+    Workload("f_sq_gt_sk_global", 1, 1, 1, 120, 70, 32, dtype="fp32", o_dtype="fp32", seed=78, window_left=5,
+             window_right=5, global_len=9),
+    Workload("f_gqa_4_1", 1, 4, 1, 65, 65, 64, dtype="fp32", o_dtype="fp32", seed=79, causal=True),
+    Workload("f_window_left_1", 1, 1, 1, 64, 64, 32, dtype="fp32", o_dtype="fp32", seed=80, causal=True, window_left=1, window_right=0),
+    Workload("f_softcap_1e12", 1, 1, 1, 127, 127, 64, dtype="fp32", o_dtype="fp32", seed=81, causal=True, softcap=1e12),
+    Workload("f_two_rows", 1, 2, 2, 2, 2, 64, dtype="fp32", o_dtype="fp32", seed=82, causal=True),
 ]
 
 
@@ -142,6 +176,32 @@ BF16_EXTRA = [
              cu_seqlens=(0, 300, 301, 512, 640, 1000, 1024), global_len=300),
     Workload("b_share_question_sigmoid", 1, 1, 1, 640, 640, 128, seed=70, causal=True, cu_seqlens=(0, 128, 384, 640),
              global_len=128, normalizer="sigmoid", o_dtype="fp32", sigmoid_bias=-math.log(640.0), std=1.5),
+    # tile-edge sizes
+    Workload("b_s2", 1, 2, 2, 2, 2, 128, seed=83, causal=True),
+    Workload("b_s64", 1, 2, 1, 64, 64, 128, seed=84, causal=True),
+    Workload("b_s65_d64", 1, 1, 1, 65, 65, 64, seed=85),
+    Workload("b_s127", 1, 1, 1, 127, 127, 128, seed=86, causal=True),
+    Workload("b_s255_d256", 1, 1, 1, 255, 255, 256, seed=87, causal=True, std=1.5),
+    Workload("b_s256", 2, 2, 2, 256, 256, 128, seed=88, causal=True),
+    Workload("b_gqa_4_1", 1, 4, 1, 300, 300, 128, seed=89, causal=True),
+    Workload("b_gqa_8", 2, 16, 2, 300, 300, 128, seed=90, causal=True, slopes=alibi_slopes(16)),
+    Workload("b_gqa_16", 1, 32, 2, 260, 260, 128, seed=91, causal=True, window_left=100, window_right=0),
+    Workload("b_gqa_3", 1, 6, 2, 300, 300, 128, seed=92, causal=True),          # odd group: one head x 256 rows per item
+    Workload("b_window_left_1", 1, 1, 1, 300, 300, 128, seed=93, causal=True, window_left=1, window_right=0),
+    Workload("b_softcap_1e12", 1, 2, 2, 300, 300, 128, seed=94, causal=True, softcap=1e12),
+    Workload("b_softcap_1e12_d256", 1, 1, 1, 300, 300, 256, seed=95, causal=True, softcap=1e12, std=1.5),
+    # D = 256, softmax with the generic score on the CTA-pair kernel: a softcap small enough takes the fixed
+    # reference (no running maximum), C * log2(e) >= 72.5, i.e. C >= 50.26, or any slope takes the running maximum
+    Workload("b_d256_softcap_50_2", 1, 2, 2, 640, 640, 256, seed=96, causal=True, softcap=50.2, std=1.5),
+    Workload("b_d256_softcap_50_3", 1, 2, 2, 640, 640, 256, seed=96, causal=True, softcap=50.3, std=1.5),
+    Workload("b_d256_softcap_100", 1, 2, 2, 900, 900, 256, seed=97, causal=True, softcap=100.0, std=2.5),
+    Workload("b_d256_softcap_slopes", 1, 2, 1, 640, 640, 256, seed=98, causal=True, softcap=30.0, slopes=(-0.5, 0.25), std=1.5),
+    Workload("b_d256_softcap_100_scores", 1, 1, 1, 640, 640, 256, seed=99, softcap=100.0, scale=1.0),
+    # more query rows than keys under masks other than plain causal
+    Workload("b_sq_gt_sk_window", 1, 2, 1, 700, 300, 128, seed=100, window_left=70, window_right=90),
+    Workload("b_sq_gt_sk_prefix_window", 1, 1, 1, 600, 330, 128, seed=101, causal=True, prefix_len=140, window_left=100, window_right=0),
+    Workload("b_sq_gt_sk_global", 1, 1, 1, 700, 400, 128, seed=102, window_left=50, window_right=50, global_len=70),
+    Workload("b_sq_gt_sk_window_d256", 1, 1, 1, 600, 260, 256, seed=103, window_left=64, window_right=64, std=1.5),
 ]
 
 
@@ -215,8 +275,9 @@ def test_host_staged_entry_point():
 
 
 # ------------------------------------------------------------------ the five benchmark configurations, full size
-def sampled_rows(w, per_head, heads, seed):
-    """Rows of a few (batch, head) pairs: the first and last tiles plus random rows."""
+def sampled_rows(w, per_head, heads, seed, every_head=0):
+    """Rows of a few (batch, head) pairs: the first and last tiles plus random rows; and ``every_head`` random
+    rows (plus the first and the last row) of EVERY (batch, head)."""
     rng = np.random.default_rng(seed)
     rows = []
     bh = [(int(rng.integers(w.B)), int(rng.integers(w.Hq))) for _ in range(heads)] + [(w.B - 1, w.Hq - 1)]
@@ -224,6 +285,10 @@ def sampled_rows(w, per_head, heads, seed):
         i = np.concatenate([np.arange(0, min(w.Sq, 130)), np.arange(max(0, w.Sq - 130), w.Sq),
                             rng.integers(0, w.Sq, size=per_head)])
         rows.append((b * w.Hq + h) * w.Sq + np.unique(i))
+    if every_head:
+        for bh_ in range(w.B * w.Hq):
+            i = np.concatenate([[0, w.Sq - 1], rng.integers(0, w.Sq, size=every_head)])
+            rows.append(bh_ * w.Sq + np.unique(i))
     return np.unique(np.concatenate(rows)).astype(np.int64)
 
 
@@ -235,7 +300,7 @@ def test_benchmark_configuration_full_size(name):
         check(w)
         return
     per_head = 96 if w.Sk <= 8192 else 24
-    check(w, rows=sampled_rows(w, per_head, 3, seed=sum(map(ord, name))))
+    check(w, rows=sampled_rows(w, per_head, 3, seed=sum(map(ord, name)), every_head=24 if w.Sk <= 8192 else 6))
 
 
 # Many short work items per CTA with the cheapest normaliser: the work-item hand-off is the busiest here.
@@ -299,3 +364,153 @@ def test_other_kernels_at_every_head_dimension(tmp_path, env_name):
     out = subprocess.run([sys.executable, str(script), root], capture_output=True, text=True, timeout=600, env=env)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-2000:]
     assert "split kernel ok" in out.stdout
+
+
+# ------------------------------------------------------------------ the paper's model configurations (Sec. 4.1)
+# Heads (Hq / Hkv / D) of the larger two models, 64/8/128 and 128/8/128: GQA groups of 8 and 16, which select the
+# two-heads-per-work-item form of the ping-pong kernel, at 16k tokens per batch with S = 1024 (B = 16) and S = 8192
+# (B = 2), for the variants of Appendix A that the benchmark configurations also use.  Compared on sampled rows of
+# every (batch, head).
+def _model_variants(base):
+    s = base.Sq
+    return [
+        base.with_(name=base.name + "_causal", causal=True),
+        base.with_(name=base.name + "_window", causal=True, window_left=511, window_right=0),
+        base.with_(name=base.name + "_alibi", causal=True, slopes=alibi_slopes(base.Hq)),
+        base.with_(name=base.name + "_softcap", causal=True, softcap=50.0),
+        base.with_(name=base.name + "_sigmoid", causal=True, normalizer="sigmoid", o_dtype="fp32",
+                   sigmoid_bias=-math.log(float(s))),
+    ]
+
+
+MODEL_SHAPES = [Workload("m64_8_s1k", 16, 64, 8, 1024, 1024, 128, seed=9100),
+                Workload("m64_8_s8k", 2, 64, 8, 8192, 8192, 128, seed=9101),
+                Workload("m128_8_s1k", 16, 128, 8, 1024, 1024, 128, seed=9102),
+                Workload("m128_8_s8k", 2, 128, 8, 8192, 8192, 128, seed=9103)]
+
+
+@pytest.mark.parametrize("base", MODEL_SHAPES, ids=lambda w: w.name)
+def test_paper_model_configurations_sampled_rows(base):
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    q, k, v = make_qkv(base)                       # one draw per shape, shared by its variants
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    tol_o, tol_l = TOL["bf16"]
+    for w in _model_variants(base):
+        rows = sampled_rows(w, 0, 0, seed=sum(map(ord, w.name)), every_head=3 if w.Sq <= 1024 else 10)
+        odt = torch.float32 if w.o_dtype == "fp32" else torch.bfloat16
+        o = torch.full((w.B, w.Hq, w.Sq, w.D), float("nan"), device=dev, dtype=odt)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        o, lse = pk.attn_fwd(qd, kd, vd, o=o, status_word=status, **pk.variant_kwargs(w, dev))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert not bool(torch.isnan(o.float()).any()), f"{w.name}: unwritten or NaN output rows"
+        o_ref, lse_ref = oracle_run(w, q, k, v, rows=rows)
+        err_o = np.abs(o.double().cpu().numpy().reshape(-1, w.D)[rows] - o_ref).max()
+        assert err_o <= tol_o, f"{w.name}: max|dO| = {err_o:.3e}"
+        if lse is not None:
+            err_l = np.abs(lse.double().cpu().numpy().reshape(-1)[rows] - lse_ref).max()
+            assert err_l <= tol_l, f"{w.name}: max|dLSE| = {err_l:.3e}"
+
+
+# ------------------------------------------------------------------ masked positions have no influence (on the GPU)
+# Large finite garbage (+-1e4) is written into K and V at a band of key positions; every query row that cannot see
+# any key of the band must come out bit-identical to the clean run (a partial tile multiplies P = 0 by whatever V
+# holds there, and the garbage scores must be masked before they reach the row maximum).
+GARBAGE_CASES = [
+    (Workload("g_causal", 1, 2, 2, 700, 700, 128, seed=110, causal=True), (450, 700)),
+    (Workload("g_causal_d256", 1, 1, 1, 640, 640, 256, seed=111, causal=True, std=1.5), (333, 640)),
+    (Workload("g_causal_d64", 1, 2, 1, 700, 700, 64, seed=112, causal=True), (129, 300)),
+    (Workload("g_window", 1, 2, 2, 900, 900, 128, seed=113, causal=True, window_left=100, window_right=0), (300, 420)),
+    (Workload("g_window_two_sided", 1, 1, 1, 900, 900, 128, seed=114, window_left=64, window_right=64), (500, 520)),
+    (Workload("g_docs", 1, 2, 2, 1024, 1024, 128, seed=115, causal=True, cu_seqlens=(0, 200, 456, 700, 1024)), (200, 456)),
+    (Workload("g_docs_bidir", 1, 1, 1, 640, 640, 256, seed=116, cu_seqlens=(0, 130, 400, 640), std=1.5), (130, 400)),
+    (Workload("g_global", 1, 2, 1, 1000, 1000, 128, seed=117, window_left=64, window_right=64, global_len=50), (400, 500)),
+    (Workload("g_share_question", 1, 1, 1, 1024, 1024, 128, seed=118, causal=True, cu_seqlens=(0, 300, 500, 800, 1024),
+              global_len=300), (500, 800)),
+    (Workload("g_prefix", 1, 1, 1, 700, 700, 128, seed=119, causal=True, prefix_len=200), (400, 700)),
+    (Workload("g_fp32_window", 1, 2, 1, 300, 300, 64, dtype="fp32", o_dtype="fp32", seed=120, causal=True, window_left=40,
+              window_right=0), (100, 160)),
+    (Workload("g_sigmoid", 1, 1, 1, 640, 640, 128, seed=121, causal=True, normalizer="sigmoid", o_dtype="fp32",
+              sigmoid_bias=-math.log(640.0)), (400, 640)),
+]
+
+
+@pytest.mark.parametrize("w,band", GARBAGE_CASES, ids=lambda x: x.name if isinstance(x, Workload) else None)
+def test_masked_positions_have_no_influence_on_the_gpu(w, band):
+    from workload_flops import row_visibility
+    q, k, v = make_qkv(w)
+    o_clean, lse_clean = gpu_run(w, q, k, v)
+    j0, j1 = band
+    rng = np.random.default_rng(w.seed)
+    sign = torch.from_numpy(rng.choice([-1.0, 1.0], size=(w.B, w.Hkv, j1 - j0, w.D)).astype(np.float32))
+    k2, v2 = k.clone(), v.clone()
+    k2[:, :, j0:j1] = (1e4 * sign).to(k.dtype)
+    v2[:, :, j0:j1] = (-1e4 * sign).to(v.dtype)
+    o_dirty, lse_dirty = gpu_run(w, q, k2, v2)
+    pre, lo, hi = row_visibility(w.Sq, w.Sk, causal=w.causal, window_left=w.window_left, window_right=w.window_right,
+                                 cu_seqlens=w.cu_seqlens, prefix_len=w.prefix_len, test_query_start=w.test_query_start,
+                                 global_len=w.global_len)
+    blind = torch.from_numpy(((hi < j0) | (lo >= j1)) & (pre <= j0))      # rows that see no key of the band
+    assert int(blind.sum()) >= 100 and int((~blind).sum()) >= 1, "the case must have rows on both sides"
+    assert torch.equal(o_clean[:, :, blind].cpu(), o_dirty[:, :, blind].cpu()), f"{w.name}: hidden keys changed O"
+    if lse_clean is not None:
+        assert torch.equal(lse_clean[:, :, blind].cpu(), lse_dirty[:, :, blind].cpu()), f"{w.name}: hidden keys changed LSE"
+    assert not torch.equal(o_clean[:, :, ~blind].cpu(), o_dirty[:, :, ~blind].cpu())     # the band is really seen elsewhere
+
+
+# ------------------------------------------------------------------ boundary: cache, device-side checks, the timeout path
+def test_tensor_map_cache_hits_and_clear():
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    w = Workload("b_cache", 1, 2, 2, 300, 300, 128, seed=122, causal=True)
+    q, k, v = (t.to(dev) for t in make_qkv(w))
+    kw = pk.variant_kwargs(w, dev)
+    o1, _ = pk.attn_fwd(q, k, v, **kw)
+    h0 = pk.cache_hits()
+    o2 = torch.empty_like(o1)
+    pk.attn_fwd(q, k, v, o=o2, **kw)
+    assert pk.cache_hits() - h0 == 3            # Q, K and V maps of the second call came from the cache
+    assert pk.clear_cache() == 0
+    h1 = pk.cache_hits()
+    o3 = torch.empty_like(o1)
+    pk.attn_fwd(q, k, v, o=o3, **kw)
+    assert pk.cache_hits() == h1                # emptied: encoded again
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2) and torch.equal(o1, o3)
+
+
+@pytest.mark.parametrize("D,dtype", [(128, "bf16"), (256, "bf16"), (64, "fp32")])
+def test_malformed_offsets_are_reported_in_the_status_word(D, dtype):
+    """cu_seqlens lives in device memory, so the host cannot check it: the kernel reports a table that decreases, does
+    not start at 0 or does not end at Sq as ATTN_ERR_DESC (5), and stays memory safe."""
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    for cu in [(0, 200, 150, 300), (3, 100, 300), (0, 100, 280)]:
+        w = Workload("b_bad_cu", 1, 2, 2, 300, 300, D, dtype=dtype, o_dtype=dtype, seed=123, causal=True, cu_seqlens=cu)
+        q, k, v = (t.to(dev) for t in make_qkv(w))
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        pk.attn_fwd(q, k, v, status_word=status, **pk.variant_kwargs(w, dev))
+        torch.cuda.synchronize()
+        assert int(status.item()) == 5, (cu, int(status.item()))
+    w = Workload("b_good_cu", 1, 2, 2, 300, 300, D, dtype=dtype, o_dtype=dtype, seed=123, causal=True, cu_seqlens=(0, 100, 100, 300))
+    check(w)                                    # an empty document is legal
+
+
+def test_bounded_wait_that_runs_out_reports_and_leaves_the_context_usable():
+    """The kernels' failure path, in its harmless form: a wait with a 1 ms limit on a barrier that nothing arrives on
+    gives up, reports ATTN_ERR_TIMEOUT (7), a second waiter on the same barrier leaves at once, the kernel ends, and
+    the next attention call on the same context is correct."""
+    import time
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    second = torch.zeros(1, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    assert pk.selftest_timeout(status, 1_000_000, second) == 0
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert int(status.item()) == 7 and int(second.item()) == 2
+    assert dt < 0.5, f"the kernel took {dt:.3f} s for a 1 ms limit"
+    check(Workload("b_after_timeout", 1, 2, 2, 300, 300, 128, seed=124, causal=True))

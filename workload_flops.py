@@ -1,5 +1,9 @@
 """Unmasked work of an attention problem: visible (query, key) pairs and the FLOPs they cost.
 
+Bookkeeping for the benchmark and the tests (it counts pairs from the mask parameters of a workload; it holds
+none of the attention arithmetic and loads no compiled library, so both the CUDA arm and the CPU-oracle arm of
+the benchmark can use it).
+
 Every mask this library builds (causal, window, same document, PrefixLM, the test-query
 clause of the causal blockwise mask) leaves each query row one contiguous key interval
 [lo(i), hi(i)], so the count is a sum of interval lengths.  4*D FLOPs per visible pair
@@ -48,7 +52,7 @@ def row_visibility(Sq: int, Sk: int, causal: bool = False, window_left: Optional
         lo = np.where(isolated, np.maximum(lo, cu[d]), lo)
         hi = np.where(isolated, np.minimum(hi, cu[d + 1] - 1), hi)
     pre = np.zeros(Sq, dtype=np.int64)
-    if global_len:
+    if global_len is not None:
         g = min(int(global_len), Sk)
         hi_causal = np.full(Sq, Sk - 1, dtype=np.int64)
         if causal:
