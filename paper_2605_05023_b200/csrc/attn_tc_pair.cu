@@ -420,7 +420,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         // between the two groups and the rescaling of O are not needed at all.
         const bool fixed_max = (SCORE == kScoreGeneric) && p.softcap > 0.f && p.slopes == nullptr && p.softcap * kLog2e < 72.5f;
         if (fixed_max) m_used = p.softcap * kLog2e - 32.0f;
-        float l_exact = 0.f;                                 // fixed reference only: sum of the unrounded weights
+        // D = 256, and always with the fixed reference: the row sum that normalises O is taken over the bf16-rounded
+        // weights that P V uses, so that O is an exactly normalised average of V rows (the rounding of a dominant
+        // weight would otherwise show in O); the LSE uses a second sum over the unrounded weights.
+        const bool rounded_sum = fixed_max || D == 256;
+        float l_exact = 0.f;                                 // rounded_sum only: sum of the unrounded weights
 
         for (int n = 0; n < niter; ++n, ++g) {
             const int kv0 = (tr.jlo + n) * kBN;
@@ -513,6 +517,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         ptx::tc_fence_after_sync();
                         const float alpha = (m_new == -INFINITY) ? 1.0f : ptx::ex2_approx(m_used - m_new);
                         l *= alpha;
+                        l_exact *= alpha;
                         m_used = m_new;
 #pragma unroll
                         for (int c = 0; c < kOC / 32; ++c) {
@@ -532,7 +537,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 #pragma unroll
                 for (int cc = 0; cc < kWgCols / 32; ++cc) {
                     uint32_t pk[16];
-                    if (fixed_max) exp_chunk<SCORE, true>(&y[cc * 32], cs, neg_m, sum2, pk, sume);
+                    if (rounded_sum) exp_chunk<SCORE, true>(&y[cc * 32], cs, neg_m, sum2, pk, sume);
                     else exp_chunk<SCORE, false>(&y[cc * 32], cs, neg_m, sum2, pk);
                     ptx::tmem_st_32x16(ts + cc * 16, pk);
                 }
@@ -540,7 +545,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 ptx::unpack2(ptx::add2(sum2[0], sum2[1]), s0, s1);
                 ptx::unpack2(ptx::add2(sum2[2], sum2[3]), s2, s3);
                 l += (s0 + s1) + (s2 + s3);
-                if (fixed_max) {
+                if (rounded_sum) {
                     ptx::unpack2(ptx::add2(sume[0], sume[1]), s0, s1);
                     l_exact += s0 + s1;
                 }
@@ -561,7 +566,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             l_row = l + l_other;
         }
         float l_lse = l_row;                                 // the LSE is the log of the sum of the unrounded weights
-        if (fixed_max) {
+        if (!SIGMOID && !RELU && rounded_sum) {
             float le_other;
             if (!exchange(l_exact, le_other)) return;
             l_lse = l_exact + le_other;

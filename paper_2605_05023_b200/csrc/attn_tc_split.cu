@@ -421,6 +421,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         if constexpr (SCORE != kScorePlain) sc = make_score_consts(p.scale, p.softcap, p.slopes ? __ldg(p.slopes + it.h) : 0.f);
         const int niter = tile_count(tr);
         float m_used = -INFINITY, l = 0.f;                   // l: this group's share of the row sum
+        // D = 256 (values of larger magnitude, 256 columns per row): the row sum that normalises O is taken over the
+        // bf16-rounded weights that P V uses, so that O is an exactly normalised average of V rows (the rounding of a
+        // dominant weight would otherwise show in O); the LSE uses a second, unrounded sum.
+        constexpr bool kRoundedSum = (D == 256);
+        float l_exact = 0.f;
 
         for (int n = 0; n < niter; ++n, ++g) {
             const int kv0 = tile_at(tr, n) * kBN;
@@ -511,6 +516,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         ptx::tc_fence_after_sync();
                         const float alpha = (m_new == -INFINITY) ? 1.0f : ptx::ex2_approx(m_used - m_new);
                         l *= alpha;
+                        l_exact *= alpha;
                         m_used = m_new;
 #pragma unroll
                         for (int c = 0; c < kOC / 32; ++c) {
@@ -525,16 +531,21 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 }
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
                 uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
+                uint64_t sume[2] = {0ull, 0ull};
 #pragma unroll
                 for (int cc = 0; cc < kWgCols / 32; ++cc) {
                     uint32_t pk[16];
-                    exp_chunk<SCORE>(&y[cc * 32], cs, neg_m, sum2, pk);
+                    exp_chunk<SCORE, kRoundedSum>(&y[cc * 32], cs, neg_m, sum2, pk, sume);
                     ptx::tmem_st_32x16(ts + cc * 16, pk);
                 }
                 float s0, s1, s2, s3;
                 ptx::unpack2(ptx::add2(sum2[0], sum2[1]), s0, s1);
                 ptx::unpack2(ptx::add2(sum2[2], sum2[3]), s2, s3);
                 l += (s0 + s1) + (s2 + s3);
+                if constexpr (kRoundedSum) {
+                    ptx::unpack2(ptx::add2(sume[0], sume[1]), s0, s1);
+                    l_exact += s0 + s1;
+                }
             }
             warp_arrive_after_tmem_st(ptx::smem_u32(&bars->p_full[buf]));
         }
@@ -547,6 +558,12 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             float l_other;
             if (!exchange(l, l_other)) return;
             l_row = l + l_other;
+        }
+        float l_lse = l_row;                                 // the LSE is the log of the sum of the unrounded weights
+        if constexpr (!SIGMOID && !RELU && kRoundedSum) {
+            float le_other;
+            if (!exchange(l_exact, le_other)) return;
+            l_lse = l_exact + le_other;
         }
         if (niter > 0) {
             // pv_done cannot serve here: the MMA thread may lag two key tiles behind, and a parity wait only
@@ -596,7 +613,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             }
         }
         if (!SIGMOID && !RELU && wg == 0 && p.lse && store_row)
-            p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = (l_row > 0.f) ? (m_used + ptx::lg2_approx(l_row)) * kLn2 : -INFINITY;
+            p.lse[((long long)it.b * p.Hq + it.h) * p.Sq + row] = (l_lse > 0.f) ? (m_used + ptx::lg2_approx(l_lse)) * kLn2 : -INFINITY;
 
 
         // Next work item: one lane reads the fetched index and shares it with the warp.

@@ -32,17 +32,17 @@ def gpu_run(w, q, k, v, poison=True):
 
 def relu_row_bounds(w, v, o_ref, p_ref):
     """Per-element error bound of the ReLU normaliser, scaled by what each ROW holds (a row of small outputs
-    gets a small bound).  O_id = sum_j P_ij V_jd with P rounded to bf16 before the product (relative error up
-    to 2^-9 per weight, independent signs: standard deviation 2^-9 / sqrt(3) * sqrt(sum_j (P_ij V_jd)^2), taken
-    at six sigma = 2^-7) and O rounded once to the output type (2^-9 relative for bf16).  fp32 inputs: every
-    step is fp32, 1e-5 of the same two row quantities."""
+    gets a small bound).  O_id = sum_j P_ij V_jd with P rounded to bf16 before the product (8 significant bits:
+    relative error up to 2^-8 per weight, independent signs: standard deviation at most 2^-8 / sqrt(3) *
+    sqrt(sum_j (P_ij V_jd)^2), taken at six sigma < 2^-6) and O rounded once to the output type (2^-8 relative
+    for bf16).  fp32 inputs: every step is fp32, 1e-5 of the same two row quantities."""
     B, Hq, Sq, D = o_ref.shape
     g = Hq // w.Hkv
     v2 = (v.double().numpy() ** 2).repeat(g, axis=1)                      # [B, Hq, Sk, D]
     spread = np.sqrt(np.einsum("bhij,bhjd->bhid", p_ref ** 2, v2))
     if w.dtype == "bf16":
-        out_round = 2.0 ** -9 if w.o_dtype == "bf16" else 2.0 ** -23
-        return 2.0 ** -7 * spread + out_round * np.abs(o_ref) + 1e-30
+        out_round = 2.0 ** -8 if w.o_dtype == "bf16" else 2.0 ** -23
+        return 2.0 ** -6 * spread + out_round * np.abs(o_ref) + 1e-30
     return 1e-5 * (spread + np.abs(o_ref)) + 1e-30
 
 
@@ -75,7 +75,8 @@ def check(w, rows=None):
     assert err_o <= tol_o, f"{w.name}: max|dO| = {err_o:.3e} > {tol_o}"
     if l_np is not None:
         both_inf = np.isneginf(l_np) & np.isneginf(lse_ref)
-        err_l = np.abs(np.where(both_inf, 0.0, l_np - lse_ref)).max()
+        with np.errstate(invalid="ignore"):           # -inf - -inf of rows with no visible key
+            err_l = np.abs(np.where(both_inf, 0.0, l_np - lse_ref)).max()
         assert err_l <= tol_l, f"{w.name}: max|dLSE| = {err_l:.3e} > {tol_l}"
     return float(err_o)
 
@@ -194,7 +195,7 @@ BF16_EXTRA = [
     # reference (no running maximum), C * log2(e) >= 72.5, i.e. C >= 50.26, or any slope takes the running maximum
     Workload("b_d256_softcap_50_2", 1, 2, 2, 640, 640, 256, seed=96, causal=True, softcap=50.2, std=1.5),
     Workload("b_d256_softcap_50_3", 1, 2, 2, 640, 640, 256, seed=96, causal=True, softcap=50.3, std=1.5),
-    Workload("b_d256_softcap_100", 1, 2, 2, 900, 900, 256, seed=97, causal=True, softcap=100.0, std=2.5),
+    Workload("b_d256_softcap_100", 1, 2, 2, 900, 900, 256, seed=97, causal=True, softcap=100.0, scale=0.5),
     Workload("b_d256_softcap_slopes", 1, 2, 1, 640, 640, 256, seed=98, causal=True, softcap=30.0, slopes=(-0.5, 0.25), std=1.5),
     Workload("b_d256_softcap_100_scores", 1, 1, 1, 640, 640, 256, seed=99, softcap=100.0, scale=1.0),
     # more query rows than keys under masks other than plain causal
@@ -416,28 +417,33 @@ def test_paper_model_configurations_sampled_rows(base):
 # ------------------------------------------------------------------ masked positions have no influence (on the GPU)
 # Large finite garbage (+-1e4) is written into K and V at a band of key positions; every query row that cannot see
 # any key of the band must come out bit-identical to the clean run (a partial tile multiplies P = 0 by whatever V
-# holds there, and the garbage scores must be masked before they reach the row maximum).
+# holds there, and the garbage scores must be masked before they reach the row maximum).  The bands are chosen so
+# that the rows that do see the band fill whole warps of 32 rows: the online softmax decides per warp when to
+# rescale the accumulator (the TMEM accesses are warp collective), so a row that shares a warp with a row whose
+# maximum jumped gets rescaled by its own, correct, factor at a different step than in the clean run and may
+# differ in the last bit; the last case has such a shared warp and is held to a few bf16 units instead.
 GARBAGE_CASES = [
-    (Workload("g_causal", 1, 2, 2, 700, 700, 128, seed=110, causal=True), (450, 700)),
-    (Workload("g_causal_d256", 1, 1, 1, 640, 640, 256, seed=111, causal=True, std=1.5), (333, 640)),
-    (Workload("g_causal_d64", 1, 2, 1, 700, 700, 64, seed=112, causal=True), (129, 300)),
-    (Workload("g_window", 1, 2, 2, 900, 900, 128, seed=113, causal=True, window_left=100, window_right=0), (300, 420)),
-    (Workload("g_window_two_sided", 1, 1, 1, 900, 900, 128, seed=114, window_left=64, window_right=64), (500, 520)),
-    (Workload("g_docs", 1, 2, 2, 1024, 1024, 128, seed=115, causal=True, cu_seqlens=(0, 200, 456, 700, 1024)), (200, 456)),
-    (Workload("g_docs_bidir", 1, 1, 1, 640, 640, 256, seed=116, cu_seqlens=(0, 130, 400, 640), std=1.5), (130, 400)),
-    (Workload("g_global", 1, 2, 1, 1000, 1000, 128, seed=117, window_left=64, window_right=64, global_len=50), (400, 500)),
-    (Workload("g_share_question", 1, 1, 1, 1024, 1024, 128, seed=118, causal=True, cu_seqlens=(0, 300, 500, 800, 1024),
-              global_len=300), (500, 800)),
-    (Workload("g_prefix", 1, 1, 1, 700, 700, 128, seed=119, causal=True, prefix_len=200), (400, 700)),
+    (Workload("g_causal", 1, 2, 2, 700, 700, 128, seed=110, causal=True), (448, 700), True),
+    (Workload("g_causal_d256", 1, 1, 1, 640, 640, 256, seed=111, causal=True, std=1.5), (352, 640), True),
+    (Workload("g_causal_d64", 1, 2, 1, 700, 700, 64, seed=112, causal=True), (160, 300), True),
+    (Workload("g_window", 1, 2, 2, 900, 900, 128, seed=113, causal=True, window_left=100, window_right=0), (288, 412), True),
+    (Workload("g_window_two_sided", 1, 1, 1, 900, 900, 128, seed=114, window_left=64, window_right=64), (512, 544), True),
+    (Workload("g_docs", 1, 2, 2, 1024, 1024, 128, seed=115, causal=True, cu_seqlens=(0, 192, 448, 700, 1024)), (192, 448), True),
+    (Workload("g_docs_bidir", 1, 1, 1, 640, 640, 256, seed=116, cu_seqlens=(0, 128, 416, 640), std=1.5), (128, 416), True),
+    (Workload("g_global", 1, 2, 1, 1000, 1000, 128, seed=117, window_left=64, window_right=64, global_len=64), (512, 544), True),
+    (Workload("g_share_question", 1, 1, 1, 1024, 1024, 128, seed=118, causal=True, cu_seqlens=(0, 320, 512, 800, 1024),
+              global_len=320), (512, 800), True),
+    (Workload("g_prefix", 1, 1, 1, 700, 700, 128, seed=119, causal=True, prefix_len=200), (416, 700), True),
     (Workload("g_fp32_window", 1, 2, 1, 300, 300, 64, dtype="fp32", o_dtype="fp32", seed=120, causal=True, window_left=40,
-              window_right=0), (100, 160)),
+              window_right=0), (100, 160), True),
     (Workload("g_sigmoid", 1, 1, 1, 640, 640, 128, seed=121, causal=True, normalizer="sigmoid", o_dtype="fp32",
-              sigmoid_bias=-math.log(640.0)), (400, 640)),
+              sigmoid_bias=-math.log(640.0)), (400, 640), True),
+    (Workload("g_causal_shared_warp", 1, 2, 2, 700, 700, 128, seed=125, causal=True), (450, 700), False),
 ]
 
 
-@pytest.mark.parametrize("w,band", GARBAGE_CASES, ids=lambda x: x.name if isinstance(x, Workload) else None)
-def test_masked_positions_have_no_influence_on_the_gpu(w, band):
+@pytest.mark.parametrize("w,band,exact", GARBAGE_CASES, ids=lambda x: x.name if isinstance(x, Workload) else None)
+def test_masked_positions_have_no_influence_on_the_gpu(w, band, exact):
     from workload_flops import row_visibility
     q, k, v = make_qkv(w)
     o_clean, lse_clean = gpu_run(w, q, k, v)
@@ -451,11 +457,24 @@ def test_masked_positions_have_no_influence_on_the_gpu(w, band):
     pre, lo, hi = row_visibility(w.Sq, w.Sk, causal=w.causal, window_left=w.window_left, window_right=w.window_right,
                                  cu_seqlens=w.cu_seqlens, prefix_len=w.prefix_len, test_query_start=w.test_query_start,
                                  global_len=w.global_len)
-    blind = torch.from_numpy(((hi < j0) | (lo >= j1)) & (pre <= j0))      # rows that see no key of the band
-    assert int(blind.sum()) >= 100 and int((~blind).sum()) >= 1, "the case must have rows on both sides"
-    assert torch.equal(o_clean[:, :, blind].cpu(), o_dirty[:, :, blind].cpu()), f"{w.name}: hidden keys changed O"
-    if lse_clean is not None:
-        assert torch.equal(lse_clean[:, :, blind].cpu(), lse_dirty[:, :, blind].cpu()), f"{w.name}: hidden keys changed LSE"
+    blind_np = ((hi < j0) | (lo >= j1)) & (pre <= j0)                     # rows that see no key of the band
+    assert int(blind_np.sum()) >= 100 and int((~blind_np).sum()) >= 1, "the case must have rows on both sides"
+    if exact and w.dtype == "bf16" and w.normalizer == "softmax":
+        # rows of a warp (32 consecutive rows of a 128-row tile) are all blind or all not
+        per_warp = blind_np[: (w.Sq // 32) * 32].reshape(-1, 32)
+        assert bool(np.all(per_warp.all(axis=1) | (~per_warp).all(axis=1))), "band not aligned to warps"
+    blind = torch.from_numpy(blind_np)
+    oc, od = o_clean[:, :, blind].cpu(), o_dirty[:, :, blind].cpu()
+    if exact:
+        assert torch.equal(oc, od), f"{w.name}: hidden keys changed O"
+        if lse_clean is not None:
+            assert torch.equal(lse_clean[:, :, blind].cpu(), lse_dirty[:, :, blind].cpu()), f"{w.name}: hidden keys changed LSE"
+    else:
+        # a rescale at another step shifts the reference of the exponentials by a non-integer power of two, so the
+        # bf16 weights round differently: the two runs agree like two correct runs (half the parity bound), while
+        # garbage of 1e4 leaking with a weight of only 1e-5 would already move O by 1e-1
+        assert float((oc.float() - od.float()).abs().max()) <= 1e-2, f"{w.name}: hidden keys changed O"
+        assert float((lse_clean[:, :, blind] - lse_dirty[:, :, blind]).abs().max()) <= 1e-3
     assert not torch.equal(o_clean[:, :, ~blind].cpu(), o_dirty[:, :, ~blind].cpu())     # the band is really seen elsewhere
 
 
