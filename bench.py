@@ -397,6 +397,8 @@ def run_sweep(args):
     rows = []
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     for w in paper_sweep_workloads():
+        if args.sweep_filter and not any(f in w.name for f in args.sweep_filter.split(",")):
+            continue
         key = (w.Hq, w.Hkv, w.D)
         if key not in bufs:
             bufs.clear()
@@ -443,6 +445,7 @@ def main():
     ap.add_argument("--no-per-config", action="store_true", help="skip the per-configuration roofline block")
     ap.add_argument("--per-config-launches", type=int, default=60)
     ap.add_argument("--sweep", choices=["paper"], help="time the paper-shaped sweep instead (one JSON object; 1 GPU)")
+    ap.add_argument("--sweep-filter", default="", help="comma-separated substrings: only sweep points whose name holds one of them")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)

@@ -46,6 +46,7 @@ namespace {
 using namespace tc;
 
 constexpr int kItemWords = 21;                   // {handed over} + the 20 words of a work item, as published in shared memory
+constexpr int kMaxOrdered = 1024;                // query blocks per head that the weight-ordered work list covers
 
 
 template <int D, int NQ>
@@ -57,7 +58,8 @@ struct Cfg {
     static constexpr int kQBytes = kBM * D * 2;
     static constexpr int kDataBytes = NQ * kQBytes + kStages * kSlotBytes;
     static constexpr int kBarBytes = 1024;
-    static constexpr int kSmemBytes = kDataBytes + kBarBytes + 1024;    // + slack to align the base to 1024
+    static constexpr int kOrderBytes = 2 * kMaxOrdered * 2;             // query-block order and weights (packed documents)
+    static constexpr int kSmemBytes = kDataBytes + kBarBytes + kOrderBytes + 1024;    // + slack to align the base to 1024
     // Softmax warpgroups first, then one warpgroup holding the producer, MMA and scheduler warps.
     // With NQ = 2 setmaxnreg moves registers from that last warpgroup to the softmax groups.
     static constexpr int kThreads = NQ * 128 + 128;
@@ -125,8 +127,10 @@ __device__ __forceinline__ TileRange tile_range(const AttnParams& p, int q0, int
 // Work item of a linear index.  Heads are taken in sections whose K/V fit in L2; inside a section the
 // query block index is the slow coordinate and runs from the last block (most keys under a causal mask)
 // to the first, so the hardware hands out the heaviest items first.
+// `order`, when not null, lists the query blocks of a head heaviest first (packed documents, see build_block_order);
+// otherwise the blocks are taken from the last to the first.
 template <int NQ>
-__device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
+__device__ __forceinline__ Item decode_item(const AttnParams& p, int lin, const uint16_t* order) {
     // The two query tiles of an item share every K / V tile.  With an even GQA group they are the same 128 rows
     // of two neighbouring query heads of one KV group (identical key ranges: no step in which only one of them
     // has work); otherwise they are 256 consecutive rows of one head (under a causal mask the second tile then
@@ -142,7 +146,7 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
     const int r = lin - sec * per_sec;
     const int sec_start = sec * sec_units;
     const int sh = min(sec_units, bh_total - sec_start);
-    const int qb = nqb - 1 - r / sh;
+    const int qb = order ? (int)order[r / sh] : nqb - 1 - r / sh;
     const int bh = sec_start + r % sh;
     const int hq_units = p.Hq / units;
     Item it;
@@ -168,6 +172,43 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
 
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barriers* bars, int32_t* status_word) {
     return bounded_wait_on<false>(bar, parity, &bars->abort_flag, status_word);
+}
+
+// Packed documents (Appendix A.2, causal blockwise mask): the number of key tiles of a query block follows its
+// position inside its document, not its index, so "last block first" is no longer "heaviest first" and the grid
+// would end with a few long items on a few SMs.  Every CTA builds the same heaviest-first order of the query
+// blocks once, in shared memory, before its roles start: weight = key tiles of the block's work item; rank =
+// blocks that are heavier, plus equally heavy blocks of lower index (a stable counting of all pairs, spread over
+// the CTA's threads, with no atomics, so that all CTAs agree on the order).  The order is used when the mask has a
+// document clause and there are at most kMaxOrdered blocks.
+template <int NQ>
+__device__ __forceinline__ bool has_block_order(const AttnParams& p) {
+    const int rows = p.head_pair ? kBM : NQ * kBM;
+    return (p.mask_flags & kMaskDocument) && (p.Sq + rows - 1) / rows <= kMaxOrdered;
+}
+template <int NQ>
+__device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* order, uint16_t* weight) {   // (its own registers)
+    const int rows = p.head_pair ? kBM : NQ * kBM;
+    const int nqb = (p.Sq + rows - 1) / rows;
+    if (!has_block_order<NQ>(p)) return;
+    for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
+        int jlo = 0x7fffffff, jhi = 0;
+        for (int t = 0; t < (p.head_pair ? 1 : NQ); ++t) {
+            const TileBounds tb = tile_bounds(p, qb * rows + t * kBM, kBM);
+            if (tb.any) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
+        }
+        weight[qb] = (uint16_t)min(max(jhi - jlo, 0), 65535);
+    }
+    __syncthreads();
+    for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
+        const int w = weight[qb];
+        int rank = 0;
+        for (int o = 0; o < nqb; ++o) {
+            const int wo = weight[o];
+            rank += (wo > w || (wo == w && o < qb)) ? 1 : 0;
+        }
+        order[rank] = (uint16_t)qb;
+    }
 }
 
 // Waits for the next work item published by the scheduler thread, copies it and (kRelease) releases it.  The
@@ -197,13 +238,15 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
 // ordinary stores for the other roles, so that no role spends time on index arithmetic and mask intervals.
 template <int NQ>
 __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* bars) {
+    // the heaviest-first order of the query blocks sits right behind the barrier block (see build_block_order)
+    const uint16_t* order = has_block_order<NQ>(p) ? reinterpret_cast<const uint16_t*>(reinterpret_cast<const uint8_t*>(bars) + 1024) : nullptr;
     int32_t* status_word = p.status_word;
     uint32_t clc_phase = 0, empty_phase = 0;
     auto publish = [&](bool got, int lin) {
         volatile int* m = bars->item_msg;
         m[0] = got ? 1 : 0;
         if (got) {
-            const Item it = decode_item<NQ>(p, lin);
+            const Item it = decode_item<NQ>(p, lin, order);
             m[1] = it.q0t[0]; m[2] = it.q0t[1]; m[3] = it.ht[0]; m[4] = it.ht[1]; m[17] = it.b; m[18] = it.g;
             m[5] = it.tr[0].jlo; m[6] = it.tr[0].jhi; m[7] = it.tr[1].jlo; m[8] = it.tr[1].jhi;
             m[9] = it.lo_max[0]; m[10] = it.hi_min[0]; m[11] = it.lo_max[1]; m[12] = it.hi_min[1];
@@ -756,6 +799,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     if (warp == 0) {
         ptx::tmem_alloc<C::kTmemCols>(ptx::smem_u32(&bars->tmem_base));
         ptx::tmem_relinquish();
+    }
+    static_assert(C::kBarBytes == 1024, "scheduler_role finds the block order 1024 bytes behind the barriers");
+    {
+        uint16_t* order = reinterpret_cast<uint16_t*>(smem + C::kDataBytes + C::kBarBytes);
+        build_block_order<NQ>(p, order, order + kMaxOrdered);
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
