@@ -105,7 +105,10 @@ typedef struct attn_variant_desc {
     int32_t* status_word;      /* optional device int32, zeroed by the caller (the library never clears it): a kernel
                                   that gives up a bounded wait stores ATTN_ERR_TIMEOUT here; a cu_seqlens table that
                                   does not start at 0, end at Sq or that decreases somewhere is reported as
-                                  ATTN_ERR_DESC (the kernel stays memory safe and the output is unspecified) */
+                                  ATTN_ERR_DESC (the kernel stays memory safe and the output is unspecified); with
+                                  the sigmoid normaliser on the CTA-pair kernel (D = 256) V is converted to fp16 on
+                                  chip, and a |v| of 65536 or more (or a non-finite v) is reported as
+                                  ATTN_ERR_UNSUPPORTED (output unspecified) */
 } attn_variant_desc;
 
 /*

@@ -23,10 +23,11 @@ constexpr float kRescaleThreshold = 8.0f;        // log2 units: P stays below 2^
 // Score instances compiled per kernel: no modifier, linear bias only, anything (softcap and / or bias).
 enum : int { kScorePlain = 0, kScoreBias = 1, kScoreGeneric = 2 };
 
-// Instruction descriptor of tcgen05.mma kind::f16: bf16 x bf16 -> fp32, A K-major.  (A and B must have the
-// same element type: an f16 A operand with a bf16 B operand is rejected by the hardware.)
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) |
+// Instruction descriptor of tcgen05.mma kind::f16: bf16 x bf16 -> fp32 (or, with f16_operands, f16 x f16 -> fp32),
+// A K-major.  (A and B must have the same element type: an f16 A operand with a bf16 B operand is rejected by
+// the hardware.)
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major, bool f16_operands = false) {
+    return (1u << 4) | (f16_operands ? 0u : ((1u << 7) | (1u << 10))) | (b_mn_major ? (1u << 16) : 0u) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 

@@ -19,6 +19,11 @@
 // Cross-CTA signalling: TMA loads of both CTAs count their bytes on the leader's `full` / `q_full`
 // barriers; tcgen05.commit arrives on the same barrier of both CTAs; the softmax warps of both CTAs
 // arrive on the leader's `p_full` / `o_free` barriers through the shared::cluster window.
+// Sigmoid normaliser (Appendix A.3): the weights are not normalised per row, so the 8 significant bits of a bf16
+// P show in O; P is written as fp16 (11 bits, scaled by 2^10 away from fp16's subnormals) and, because
+// tcgen05.mma wants A and B of one type, every V tile is converted from bf16 to fp16 in shared memory, in place,
+// by a fourth warpgroup of each CTA once its TMA load has landed (exact for |v| < 65536; anything larger is
+// reported as ATTN_ERR_UNSUPPORTED in the status word).  P V is then one pass over fp16 operands.
 // Every mbarrier wait is bounded (see bounded_wait); the only unbounded waits are the cluster barriers at
 // start and exit, which every thread of both CTAs reaches.
 #include <cuda.h>
@@ -54,6 +59,11 @@ struct Cfg {
     static constexpr int kProducerWarp = 8;
     static constexpr int kMmaWarp = 9;
     static constexpr int kSchedWarp = 10;
+    static constexpr int kSpareWarp = 11;
+    static constexpr int kConverterWarp = 12;                           // sigmoid instances: a fourth warpgroup turns V into fp16
+    static constexpr int kThreadsSigmoid = 512;
+    static constexpr int kRegsSoftmax = 168, kRegsOther = 80, kRegsConverter = 80;   // sigmoid instances (setmaxnreg)
+    static_assert(2 * 128 * kRegsSoftmax + 128 * kRegsOther + 128 * kRegsConverter <= 512 * 128, "register budget");
     static constexpr int kItemConsumers = kSoftmaxWarps + 3;            // local warps that read each fetched item
     static constexpr int kTmemCols = 512;
     static constexpr int kSBufs = (D == 128) ? 3 : 2;                   // S buffers: as many as fit beside O in TMEM
@@ -68,7 +78,7 @@ struct Cfg {
 struct Barriers {
     uint64_t q_full;             // L  both Q tiles landed (TMA of both CTAs)
     uint64_t q_empty;            // B  last QK^T of the item done: the Q tile may be overwritten
-    uint64_t full[kMaxStages];   // L  both halves of a ring slot landed
+    uint64_t full[kMaxStages];   // L  both halves of a ring slot landed (V of a sigmoid instance: and converted)
     uint64_t empty[kMaxStages];  // B  ring slot consumed (tcgen05.commit to both CTAs)
     uint64_t s_full[3];          // B  S buffer written by QK^T
     uint64_t p_full[3];          // L  all of P written in both CTAs (16 warp arrivals)
@@ -84,6 +94,8 @@ struct Barriers {
     uint32_t item_value[2];      // B  {got, linear CTA index of the pair's first CTA}
     uint32_t tmem_base;
     int abort_flag;
+    uint64_t landed[kMaxStages]; // B  sigmoid instances: this CTA's half of a V tile landed (TMA), ready to be converted
+    uint64_t converted;          // B  sigmoid instances: the four converter warps are done with a V slot (4 arrivals)
 };
 static_assert(sizeof(Barriers) <= 1024, "barrier block");
 
@@ -179,7 +191,7 @@ __device__ __forceinline__ void scheduler_role(Barriers* bars, int32_t* status_w
 // ------------------------------------------------------------------------------------------------
 // producer: TMA (this CTA's Q tile, its 64 keys of every K tile, its half of the columns of every V tile)
 // ------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool V_F16>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
                                               const CUtensorMap* tmap_v, const AttnParams& p, Barriers* bars,
                                               uint32_t q_smem, uint32_t ring_smem, uint32_t rank) {
@@ -193,18 +205,28 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
     int pair = (int)(blockIdx.x >> 1);
 
     // Waits for the slot to be free in this CTA; the leader arms its `full` barrier for the bytes of both CTAs.
-    auto open_slot = [&](uint32_t& dst, uint32_t& bar) -> bool {
+    // V of a sigmoid instance (V_F16): the bytes are counted on this CTA's own `landed` barrier instead; the
+    // converter warps of both CTAs complete the leader's `full` barrier (two arrivals, so a K slot adds one).
+    auto open_slot = [&](uint32_t& dst, uint32_t& bar, bool is_v) -> bool {
         if (!bounded_wait(ptx::smem_u32(&bars->empty[ps]), pph ^ 1u, bars, p.status_word)) return false;
-        bar = ptx::smem_u32(&bars->full[ps]);
         dst = ring_smem + ps * C::kSlotBytes;
-        if (rank == 0) ptx::mbar_arrive_expect_tx(bar, 2 * C::kSlotBytes);
+        if (V_F16 && is_v) {
+            bar = ptx::smem_u32(&bars->landed[ps]);
+            ptx::mbar_arrive_expect_tx(bar, C::kSlotBytes);
+        } else {
+            bar = ptx::smem_u32(&bars->full[ps]);
+            if (rank == 0) {
+                ptx::mbar_arrive_expect_tx(bar, 2 * C::kSlotBytes);
+                if (V_F16) ptx::mbar_arrive(bar);
+            }
+        }
         if (++ps == C::kStages) { ps = 0; pph ^= 1u; }
         return true;
     };
     // Keys [128 j + 64 rank, + 64) of K, all D columns: D/64 boxes of [64 keys x 64 columns].
     auto produce_k = [&](const Item& it, int j) -> bool {
         uint32_t dst, bar;
-        if (!open_slot(dst, bar)) return false;
+        if (!open_slot(dst, bar, false)) return false;
 #pragma unroll
         for (int bx = 0; bx < D / 64; ++bx)
             ptx::tma_load_4d_pair(dst + bx * (C::kBoxBytes / 2), tmap_k, bar, bx * 64, j * kBN + (int)rank * 64, it.g, it.b);
@@ -213,10 +235,12 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
     // All 128 keys of V, columns [rank D/2, + D/2): D/128 boxes of [128 keys x 64 columns].
     auto produce_v = [&](const Item& it, int j) -> bool {
         uint32_t dst, bar;
-        if (!open_slot(dst, bar)) return false;
+        if (!open_slot(dst, bar, true)) return false;
 #pragma unroll
-        for (int bx = 0; bx < D / 128; ++bx)
-            ptx::tma_load_4d_pair(dst + bx * C::kBoxBytes, tmap_v, bar, (int)rank * (D / 2) + bx * 64, j * kBN, it.g, it.b);
+        for (int bx = 0; bx < D / 128; ++bx) {
+            if constexpr (V_F16) ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_v, bar, (int)rank * (D / 2) + bx * 64, j * kBN, it.g, it.b);
+            else ptx::tma_load_4d_pair(dst + bx * C::kBoxBytes, tmap_v, bar, (int)rank * (D / 2) + bx * 64, j * kBN, it.g, it.b);
+        }
         return true;
     };
 
@@ -247,14 +271,87 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
 }
 
 // ------------------------------------------------------------------------------------------------
+// converter (sigmoid instances): a warpgroup per CTA turns each landed V tile from bf16 into fp16, in place
+// ------------------------------------------------------------------------------------------------
+// It walks the ring in the producer's order and acts on the V slots only.  bf16 -> fp16 is exact for normal
+// values below 65536 in magnitude (8 significant bits fit in 11); smaller than 2^-14 they lose bits that no
+// output can show (absolute error below 2^-25 per product).  A value of 65536 or more (or a non-finite one)
+// cannot be represented: the group reports ATTN_ERR_UNSUPPORTED in the status word.
+template <int D>
+__device__ __forceinline__ void converter_role(const AttnParams& p, Barriers* bars, uint8_t* ring_ptr) {
+    using C = Cfg<D>;
+    const int lane = threadIdx.x & 31;
+    const int cthread = threadIdx.x & 127;          // thread within the converter warpgroup
+    int ps = 0;
+    uint32_t landed_phase = 0;                      // bit s: parity of the next completion of landed[s]
+    uint32_t item_phase = 0;
+    int pair = (int)(blockIdx.x >> 1);
+    uint32_t too_large = 0;
+    uint32_t slots_done = 0;
+    const uint32_t full_on_leader = ptx::mapa(ptx::smem_u32(&bars->full[0]), 0);
+
+    auto skip_slot = [&]() { if (++ps == C::kStages) ps = 0; };
+    auto convert_slot = [&]() -> bool {
+        if (!bounded_wait(ptx::smem_u32(&bars->landed[ps]), (landed_phase >> ps) & 1u, bars, p.status_word)) return false;
+        landed_phase ^= 1u << ps;
+        uint4* slot = reinterpret_cast<uint4*>(ring_ptr + ps * C::kSlotBytes);
+#pragma unroll 4
+        for (int i = cthread; i < C::kSlotBytes / 16; i += 128) {
+            uint4 w = slot[i];
+            uint32_t* x = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                too_large = __vmaxu2(too_large, x[e] & 0x7fff7fffu);       // largest |bf16| bit pattern seen
+                x[e] = ptx::pack_f16x2(__uint_as_float(x[e] << 16), __uint_as_float(x[e] & 0xffff0000u));
+            }
+            slot[i] = w;
+        }
+        ptx::fence_proxy_async_smem();              // these generic writes come before the MMA's reads of the slot
+        // The four warps meet on a (bounded) mbarrier; the first thread then tells the leader's MMA thread.
+        warp_arrive(ptx::smem_u32(&bars->converted));
+        if (cthread == 0) {
+            if (!bounded_wait(ptx::smem_u32(&bars->converted), slots_done & 1u, bars, p.status_word)) return false;
+            ptx::mbar_arrive_cluster(full_on_leader + ps * 8);
+        }
+        ++slots_done;
+        skip_slot();
+        return true;
+    };
+
+    bool ok = true;
+    while (ok) {
+        const Item it = decode_item(p, pair);
+        const int J0 = it.tr.jlo, J1 = it.tr.jhi;
+        if (J0 < J1) {
+#pragma unroll
+            for (int t = 0; t < C::kSBufs - 1; ++t)
+                if (J0 + t < J1) skip_slot();                                   // K
+            for (int j = J0; j < J1 && ok; ++j) {
+                if (j + C::kSBufs - 1 < J1) skip_slot();                        // K
+                ok = convert_slot();                                            // V
+            }
+        }
+        if (!ok) break;
+        int got = 0;
+        if (lane == 0) got = next_item(bars, item_phase, p.status_word, pair) ? 1 : 0;
+        got = __shfl_sync(0xffffffffu, got, 0);
+        pair = __shfl_sync(0xffffffffu, pair, 0);
+        if (!got) break;
+    }
+    // 0x4780 is bf16 65536: that and everything above (infinities and NaNs included) has no fp16 counterpart
+    const bool bad = ((too_large & 0xffffu) >= 0x4780u) || ((too_large >> 16) >= 0x4780u);
+    if (__any_sync(0xffffffffu, bad) && lane == 0 && p.status_word) atomicCAS(p.status_word, 0, (int)ATTN_ERR_UNSUPPORTED);
+}
+
+// ------------------------------------------------------------------------------------------------
 // MMA issuer (one thread of the leader CTA)
 // ------------------------------------------------------------------------------------------------
-template <int D, bool P_HI_LO>
+template <int D, bool V_F16>
 __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, uint32_t tmem, uint32_t q_smem,
                                          uint32_t ring_smem) {
     using C = Cfg<D>;
     constexpr uint32_t kIdescQK = instr_desc(2 * kBM, kBN, false);
-    constexpr uint32_t kIdescPV = instr_desc(2 * kBM, D, true);
+    constexpr uint32_t kIdescPV = instr_desc(2 * kBM, D, true, V_F16);    // sigmoid instances: P and V are fp16
     // Descriptor halves (128-byte swizzle, SBO = 1024 B, sm_100 version bit): hi is constant per operand kind,
     // lo = (address >> 4) | (LBO >> 4) << 16 advances by compile-time constants inside a tile.
     constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -277,7 +374,10 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
     int pair = (int)(blockIdx.x >> 1);
 
     auto next_slot = [&](int& slot) -> bool {
-        if (!bounded_wait(bar_full + cs * 8, cph, bars, p.status_word)) return false;
+        // (V_F16: the peer's converter warp arrives on this barrier after writing its shared memory)
+        if (!(V_F16 ? bounded_wait_cluster(bar_full + cs * 8, cph, bars, p.status_word)
+                    : bounded_wait(bar_full + cs * 8, cph, bars, p.status_word)))
+            return false;
         slot = cs;
         if (++cs == C::kStages) { cs = 0; cph ^= 1u; }
         return true;
@@ -295,8 +395,8 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
         }
         ptx::tc_commit_pair(bar_s_full + buf * 8);
     };
-    // O (+)= P[buf] V over the 128 keys of the tile.  Softmax group w wrote the bf16 P of keys [64 w, 64 w + 64)
-    // over its own S columns, starting at column 64 w (+ col_off for the residual tile of the sigmoid path).
+    // O (+)= P[buf] V over the 128 keys of the tile.  Softmax group w wrote the 16-bit P of keys [64 w, 64 w + 64)
+    // over its own S columns, starting at column 64 w.
     // B operand: this CTA's D/2 columns of V for all 128 keys, D/128 boxes of [128 keys x 128 B].
     auto issue_pv = [&](int buf, int vslot, bool accumulate, uint32_t col_off) {
         const uint32_t b_lo = (ring_lo + (uint32_t)vslot * (C::kSlotBytes >> 4)) | kLoV;
@@ -338,13 +438,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
                 }
                 if (!bounded_wait(bar_p_full + buf * 8, ph, bars, p.status_word)) return;
                 ptx::tc_fence_after_sync();
-                if constexpr (P_HI_LO) {
-                    // P = P_hi + P_lo, two bf16 tiles 32 columns apart inside each group's S columns.
-                    issue_pv(buf, vslot, j > J0, 32u);
-                    issue_pv(buf, vslot, true, 0u);
-                } else {
-                    issue_pv(buf, vslot, j > J0, 0u);
-                }
+                issue_pv(buf, vslot, j > J0, 0u);
                 ptx::tc_commit_pair(bar_pv_done + buf * 8);
                 if (j == J1 - 1) ptx::tc_commit_pair(ptx::smem_u32(&bars->o_done));
                 ptx::tc_commit_pair(bar_empty + vslot * 8);
@@ -370,7 +464,7 @@ template <int D, int SCORE, int NORM>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars, float* xchg, uint32_t tmem, int wg,
                                              uint32_t rank) {
     using C = Cfg<D>;
-    constexpr bool SIGMOID = (NORM == kNormSigmoid);   // out_scale * sigmoid(s + b), P as a bf16 hi + lo pair
+    constexpr bool SIGMOID = (NORM == kNormSigmoid);   // out_scale * sigmoid(s + b), P and V as fp16
     constexpr bool RELU = (NORM == kNormRelu);         // out_scale * max(s, 0), no exponential at all
     constexpr int kOC = D / 2;                                // O columns handled by each group
     const int wg_thread = threadIdx.x & 127;                 // row within the tile
@@ -464,26 +558,24 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 
             if constexpr (SIGMOID) {
                 // Appendix A.3: p = sigmoid(s + b); a masked score (-inf) gives exactly 0.  An unnormalised row can
-                // be carried by a few large weights, so bf16 rounding of P (up to 2^-8 relative) would show in O: P is split into
-                // P_hi = bf16(p) in this group's columns [0,32) and the residual P_lo = bf16(p - P_hi) in its columns
-                // [32,64); the MMA thread accumulates both.  out_scale is applied in the epilogue.
-                const uint64_t nb2 = ptx::pack2(-sig_bias2, -sig_bias2), neg1 = ptx::pack2(-1.0f, -1.0f);
+                // be carried by a few large weights, so the 8 significant bits of a bf16 P would show in O: P is
+                // written as fp16, scaled by 2^10 (2^10 * sigmoid(x) = 1 / (2^-10 + 2^(-x log2 e - 10)): the scale
+                // rides in the constants; the epilogue takes it out again together with out_scale).
+                const uint64_t nb2 = ptx::pack2(-sig_bias2 - 10.0f, -sig_bias2 - 10.0f), neg1 = ptx::pack2(-1.0f, -1.0f);
+                constexpr float kTwoToMinus10 = 0.0009765625f;
 #pragma unroll
                 for (int cc = 0; cc < kWgCols / 32; ++cc) {
-                    uint32_t pk[16], pl[16];
+                    uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const uint64_t yy = ptx::pack2(__uint_as_float(y[cc * 32 + 2 * i]), __uint_as_float(y[cc * 32 + 2 * i + 1]));
                         float z0, z1;
-                        ptx::unpack2(ptx::fma2(yy, neg1, nb2), z0, z1);                  // -(s + b) in log2 units
-                        const float p0 = ptx::rcp_approx(1.0f + ptx::ex2_approx(z0));
-                        const float p1 = ptx::rcp_approx(1.0f + ptx::ex2_approx(z1));
-                        const uint32_t hi = ptx::pack_bf16x2(p0, p1);
-                        pk[i] = hi;
-                        pl[i] = ptx::pack_bf16x2(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
+                        ptx::unpack2(ptx::fma2(yy, neg1, nb2), z0, z1);                  // -(s + b) in log2 units, - 10
+                        const float p0 = ptx::rcp_approx(kTwoToMinus10 + ptx::ex2_approx(z0));
+                        const float p1 = ptx::rcp_approx(kTwoToMinus10 + ptx::ex2_approx(z1));
+                        pk[i] = ptx::pack_f16x2(p0, p1);
                     }
                     ptx::tmem_st_32x16(ts + cc * 16, pk);
-                    ptx::tmem_st_32x16(ts + 32 + cc * 16, pl);
                 }
             } else if constexpr (RELU) {
                 // Appendix A.3: p = max(s, 0) in log2 units (the epilogue multiplies by out_scale * ln 2); a masked
@@ -578,7 +670,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             ++items_done;
             ptx::tc_fence_after_sync();
         }
-        const float inv = SIGMOID ? p.out_scale : (RELU ? p.out_scale * kLn2 : (l_row > 0.f ? 1.0f / l_row : 0.f));
+        const float inv = SIGMOID ? p.out_scale * 0.0009765625f : (RELU ? p.out_scale * kLn2 : (l_row > 0.f ? 1.0f / l_row : 0.f));
         char* obase = reinterpret_cast<char*>(p.o) +
                       ((long long)it.b * p.os[0] + (long long)it.h * p.os[1] + (long long)row * p.os[2] + wg * kOC) * (p.o_fp32 ? 4 : 2);
 #pragma unroll
@@ -634,10 +726,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 // kernel (cluster of two CTAs)
 // ------------------------------------------------------------------------------------------------
 template <int D, int SCORE, int NORM>
-__global__ void __launch_bounds__(Cfg<D>::kThreads, 1)
+__global__ void __launch_bounds__(NORM == kNormSigmoid ? Cfg<D>::kThreadsSigmoid : Cfg<D>::kThreads, 1)
 attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                      const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnParams p) {
     using C = Cfg<D>;
+    constexpr bool kVF16 = (NORM == kNormSigmoid);     // P and V as fp16 (see the top of this file)
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t base = ptx::smem_u32(smem);
     const uint32_t rank = ptx::cluster_ctarank();
@@ -666,12 +759,14 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
         }
         for (int t = 0; t < 2; ++t) ptx::mbar_init(ptx::smem_u32(&bars->xchg[t]), C::kSoftmaxWarps);
         for (int s = 0; s < kMaxStages; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&bars->full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&bars->landed[s]), 1);
+            if (s == 0) ptx::mbar_init(ptx::smem_u32(&bars->converted), 4);
+            ptx::mbar_init(ptx::smem_u32(&bars->full[s]), kVF16 ? 2 : 1);   // sigmoid: two arrivals per use (see open_slot)
             ptx::mbar_init(ptx::smem_u32(&bars->empty[s]), 1);
         }
         ptx::mbar_init(ptx::smem_u32(&bars->clc), 1);
         ptx::mbar_init(ptx::smem_u32(&bars->item_full), 1);
-        ptx::mbar_init(ptx::smem_u32(&bars->item_empty), rank == 0 ? C::kItemConsumers : C::kItemConsumers - 1);   // no MMA thread on the peer
+        ptx::mbar_init(ptx::smem_u32(&bars->item_empty), (rank == 0 ? C::kItemConsumers : C::kItemConsumers - 1) + (kVF16 ? 4 : 0));   // no MMA thread on the peer; sigmoid: four converter warps
         ptx::mbar_init(ptx::smem_u32(&bars->item_ready), 2);
         bars->abort_flag = 0;
         ptx::fence_mbar_init();
@@ -687,15 +782,20 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(&bars->tmem_base);
 
     if (warp < C::kSoftmaxWarps) {
+        if constexpr (kVF16) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
         softmax_role<D, SCORE, NORM>(p, bars, xchg, tmem, warp >> 2, rank);
+    } else if (kVF16 && warp >= C::kConverterWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsConverter));
+        converter_role<D>(p, bars, smem + C::kQBytes);
     } else {
+        if constexpr (kVF16) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         if (warp == C::kProducerWarp) {
-            if (lane == 0) producer_role<D>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem, rank);
+            if (lane == 0) producer_role<D, kVF16>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem, rank);
         } else if (warp == C::kMmaWarp) {
-            if (lane == 0 && rank == 0) mma_role<D, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
+            if (lane == 0 && rank == 0) mma_role<D, kVF16>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
             if (lane == 0) scheduler_role(bars, p.status_word, rank);
-        } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
+        } else if (warp == C::kSpareWarp && blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
             check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
         __syncwarp();
@@ -741,7 +841,7 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(C::kThreads, 1, 1);
+    cfg.blockDim = dim3(NORM == kNormSigmoid ? C::kThreadsSigmoid : C::kThreads, 1, 1);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];

@@ -533,3 +533,32 @@ def test_bounded_wait_that_runs_out_reports_and_leaves_the_context_usable():
     assert int(status.item()) == 7 and int(second.item()) == 2
     assert dt < 0.5, f"the kernel took {dt:.3f} s for a 1 ms limit"
     check(Workload("b_after_timeout", 1, 2, 2, 300, 300, 128, seed=124, causal=True))
+
+
+def test_sigmoid_reports_values_of_v_that_fp16_cannot_hold():
+    """The sigmoid normaliser at D = 256 (and at D = 128 on the CTA-pair kernel) converts V to fp16 on chip: a finite
+    |v| of 65536 or more has no fp16 counterpart and is reported as ATTN_ERR_UNSUPPORTED (3) in the status word;
+    values up to the largest bf16 below that pass, and the softmax path takes any finite V."""
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    w = Workload("b_sig_big_v", 1, 1, 1, 300, 300, 256, seed=126, causal=True, normalizer="sigmoid", o_dtype="fp32",
+                 sigmoid_bias=-math.log(300.0))
+    q, k, v = make_qkv(w)
+    for big, expect in ((65280.0, 0), (65536.0, 3), (1e30, 3)):
+        v2 = v.clone()
+        v2[0, 0, 17, 5] = big
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        o, _ = pk.attn_fwd(q.to(dev), k.to(dev), v2.to(dev), status_word=status, o_dtype=torch.float32, **pk.variant_kwargs(w, dev))
+        torch.cuda.synchronize()
+        assert int(status.item()) == expect, (big, int(status.item()))
+        if expect == 0:
+            o_ref, _ = oracle_run(w, q, k, v2)
+            # rows that see key 17 carry a weight of about 1/300 of 65280: the bound scales with the output
+            assert np.abs(o.double().cpu().numpy() - o_ref).max() <= 2e-2 + 2.0 ** -11 * np.abs(o_ref).max()
+    ws = w.with_(name="b_softmax_big_v", normalizer="softmax", o_dtype="bf16")
+    v2 = v.clone()
+    v2[0, 0, 17, 5] = 1e30
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    pk.attn_fwd(q.to(dev), k.to(dev), v2.to(dev), status_word=status, **pk.variant_kwargs(ws, dev))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
