@@ -291,8 +291,15 @@ __device__ __forceinline__ void converter_role(const AttnParams& p, Barriers* ba
     const uint32_t full_on_leader = ptx::mapa(ptx::smem_u32(&bars->full[0]), 0);
 
     auto skip_slot = [&]() { if (++ps == C::kStages) ps = 0; };
+    // All 32 lanes of a warp take every decision together (the waits are made by lane 0 and shared), so that a run
+    // that is being abandoned leaves the warp-collective operations below with all their lanes.
+    auto warp_wait = [&](uint32_t bar, uint32_t parity) -> bool {
+        int ok = 1;
+        if (lane == 0) ok = bounded_wait(bar, parity, bars, p.status_word) ? 1 : 0;
+        return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    };
     auto convert_slot = [&]() -> bool {
-        if (!bounded_wait(ptx::smem_u32(&bars->landed[ps]), (landed_phase >> ps) & 1u, bars, p.status_word)) return false;
+        if (!warp_wait(ptx::smem_u32(&bars->landed[ps]), (landed_phase >> ps) & 1u)) return false;
         landed_phase ^= 1u << ps;
         uint4* slot = reinterpret_cast<uint4*>(ring_ptr + ps * C::kSlotBytes);
 #pragma unroll 4
@@ -307,12 +314,11 @@ __device__ __forceinline__ void converter_role(const AttnParams& p, Barriers* ba
             slot[i] = w;
         }
         ptx::fence_proxy_async_smem();              // these generic writes come before the MMA's reads of the slot
-        // The four warps meet on a (bounded) mbarrier; the first thread then tells the leader's MMA thread.
+        // The four warps meet on a (bounded) mbarrier: none goes on to the next slot, and the first one does not
+        // tell the leader's MMA thread, before all four are done with this one.
         warp_arrive(ptx::smem_u32(&bars->converted));
-        if (cthread == 0) {
-            if (!bounded_wait(ptx::smem_u32(&bars->converted), slots_done & 1u, bars, p.status_word)) return false;
-            ptx::mbar_arrive_cluster(full_on_leader + ps * 8);
-        }
+        if (!warp_wait(ptx::smem_u32(&bars->converted), slots_done & 1u)) return false;
+        if (cthread == 0) ptx::mbar_arrive_cluster(full_on_leader + ps * 8);
         ++slots_done;
         skip_slot();
         return true;

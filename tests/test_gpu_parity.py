@@ -313,11 +313,15 @@ SHORT_ITEMS_GLOBAL = Workload("short_items_global", 8, 16, 16, 1024, 1024, 128, 
                               global_len=64, normalizer="relu", out_scale=1.0 / 1024)
 SHORT_ITEMS_PAIR = Workload("short_items_pair", 8, 8, 8, 1024, 1024, 256, seed=72, causal=True, normalizer="relu",
                             out_scale=1.0 / 1024)
-BACK_TO_BACK_EXTRA = {w.name: w for w in (SHORT_ITEMS_RELU, SHORT_ITEMS_GLOBAL, SHORT_ITEMS_PAIR)}
+# Sigmoid normaliser on the CTA-pair kernel: the fourth warpgroup converts every V tile to fp16 between its TMA load and
+# its P V, one more hand-off per key tile; short items make the ring wrap often.
+SHORT_ITEMS_SIGMOID = Workload("short_items_sigmoid", 8, 8, 8, 1024, 1024, 256, seed=127, normalizer="sigmoid",
+                               out_scale=1.0 / 1024, std=1.5)
+BACK_TO_BACK_EXTRA = {w.name: w for w in (SHORT_ITEMS_RELU, SHORT_ITEMS_GLOBAL, SHORT_ITEMS_PAIR, SHORT_ITEMS_SIGMOID)}
 
 
-@pytest.mark.parametrize("name", ["c2_causal", "c3_gqa_window_alibi", "c4a_softcap", "short_items_relu", "short_items_global",
-                                  "short_items_pair"])
+@pytest.mark.parametrize("name", ["c2_causal", "c3_gqa_window_alibi", "c4a_softcap", "c4b_sigmoid", "c5_packed_doc_causal",
+                                  "short_items_relu", "short_items_global", "short_items_pair", "short_items_sigmoid"])
 def test_back_to_back_launches_all_report_ok(name):
     """300 launches of a full-size configuration queued without a host sync in between, each with its own
     status word: the persistent work loop (many work items per CTA, work handed out by the hardware) must
@@ -329,7 +333,7 @@ def test_back_to_back_launches_all_report_ok(name):
     kw = pk.variant_kwargs(w, dev)
     n = 300
     status = torch.zeros((n, 1), dtype=torch.int32, device=dev)
-    o_first = torch.empty((w.B, w.Hq, w.Sq, w.D), device=dev, dtype=torch.bfloat16)
+    o_first = torch.empty((w.B, w.Hq, w.Sq, w.D), device=dev, dtype=torch.float32 if w.o_dtype == "fp32" else torch.bfloat16)
     o_last = torch.empty_like(o_first)
     for i in range(n):
         pk.attn_fwd(q, k, v, o=o_first if i == 0 else o_last, status_word=status[i], **kw)
@@ -346,6 +350,21 @@ import test_gpu_parity as t
 from synth_inputs import small_workloads
 for w in small_workloads() + t.BF16_EXTRA:
     t.check(w)
+# many short work items per CTA (the ring wraps, work items are handed out by the hardware) on the forced kernel
+import torch, paper_2605_05023_b200 as pk
+from synth_inputs import Workload, make_qkv
+dev = torch.device("cuda:0")
+for w in (Workload("stress_sigmoid", 8, 16, 16, 1024, 1024, 128, seed=128, normalizer="sigmoid", out_scale=1.0 / 1024),
+          Workload("stress_softmax", 8, 16, 4, 1024, 1024, 128, seed=129, causal=True, window_left=300, window_right=0)):
+    q, k, v = (x.to(dev) for x in make_qkv(w))
+    kw = pk.variant_kwargs(w, dev)
+    status = torch.zeros((60, 1), dtype=torch.int32, device=dev)
+    outs = [torch.empty((w.B, w.Hq, w.Sq, w.D), device=dev, dtype=torch.bfloat16) for _ in range(2)]
+    for i in range(60):
+        pk.attn_fwd(q, k, v, o=outs[0 if i == 0 else 1], status_word=status[i], **kw)
+    torch.cuda.synchronize()
+    assert int(status.abs().sum().item()) == 0, status.flatten().tolist()
+    assert torch.equal(outs[0], outs[1])
 print("split kernel ok")
 """
 
