@@ -106,8 +106,8 @@ typedef struct attn_variant_desc {
                                   that gives up a bounded wait stores ATTN_ERR_TIMEOUT here; a cu_seqlens table that
                                   does not start at 0, end at Sq or that decreases somewhere is reported as
                                   ATTN_ERR_DESC (the kernel stays memory safe and the output is unspecified); with
-                                  the sigmoid normaliser on the CTA-pair kernel (D = 256) V is converted to fp16 on
-                                  chip, and a |v| of 65536 or more (or a non-finite v) is reported as
+                                  the sigmoid normaliser at D = 128 and D = 256 (CTA-pair kernel) V is converted to
+                                  fp16 on chip, and a |v| of 65536 or more (or a non-finite v) is reported as
                                   ATTN_ERR_UNSUPPORTED (output unspecified) */
 } attn_variant_desc;
 

@@ -887,7 +887,9 @@ int launch_attn_fwd_bf16_split(const AttnParams& p, cudaStream_t stream);   // a
 int launch_attn_fwd_bf16_pair(const AttnParams& p, cudaStream_t stream);    // attn_tc_pair.cu
 
 // Kernel choice.  D = 64, 128: two query tiles per work item ping-pong on one SM (this file).  D = 256: CTA pairs
-// (attn_tc_pair.cu), which halve the K / V traffic from L2.  B200ATTN_FORCE_SPLIT=1 / B200ATTN_FORCE_PAIR=1 in the
+// (attn_tc_pair.cu), which halve the K / V traffic from L2.  The sigmoid normaliser at D = 128 runs on the CTA-pair
+// kernel too: its one-pass fp16 form of P V (with V converted on chip) beats the bf16 hi + lo pair of this file by
+// 15 to 40 % on the paper-shaped sweep.  B200ATTN_FORCE_SPLIT=1 / B200ATTN_FORCE_PAIR=1 in the
 // environment route every head dimension they support to the one-tile kernel (attn_tc_split.cu) or to the
 // CTA-pair kernel; the tests use them to cover those kernels at the other head dimensions.
 int launch_attn_fwd_bf16(const AttnParams& p, cudaStream_t stream, int* launches) {
@@ -897,7 +899,7 @@ int launch_attn_fwd_bf16(const AttnParams& p, cudaStream_t stream, int* launches
     int rc;
     if (force_split || (p.mask_flags & kMaskGlobal)) {      // two key intervals per row: only the one-tile kernel walks them
         rc = launch_attn_fwd_bf16_split(p, stream);
-    } else if (p.D == 256 || (force_pair && p.D == 128)) {
+    } else if (p.D == 256 || (p.D == 128 && (force_pair || p.normalizer == kNormSigmoid))) {
         rc = launch_attn_fwd_bf16_pair(p, stream);
     } else {
         switch (p.D) {

@@ -555,7 +555,7 @@ def test_bounded_wait_that_runs_out_reports_and_leaves_the_context_usable():
 
 
 def test_sigmoid_reports_values_of_v_that_fp16_cannot_hold():
-    """The sigmoid normaliser at D = 256 (and at D = 128 on the CTA-pair kernel) converts V to fp16 on chip: a finite
+    """The sigmoid normaliser at D = 128 and D = 256 (CTA-pair kernel) converts V to fp16 on chip: a finite
     |v| of 65536 or more has no fp16 counterpart and is reported as ATTN_ERR_UNSUPPORTED (3) in the status word;
     values up to the largest bf16 below that pass, and the softmax path takes any finite V."""
     import paper_2605_05023_b200 as pk
