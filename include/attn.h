@@ -74,7 +74,7 @@ enum { ATTN_NORM_SOFTMAX = 0, ATTN_NORM_SIGMOID = 1, ATTN_NORM_RELU = 2 };   /* 
  * global_len, and every key for a query row at position i' < global_len, passes the window and document
  * clauses (Global Sliding Window: "i in G or j in G"; Share Question mask: documents = prompt and responses,
  * global_len = prompt length, with the causal clause).  With ATTN_MASK_GLOBAL a row sees up to two key
- * intervals; the bf16 path then runs on the one-tile-per-CTA tensor-core kernel. */
+ * intervals (the global keys and its own window / document). */
 enum { ATTN_MASK_CAUSAL = 1u, ATTN_MASK_WINDOW = 2u, ATTN_MASK_DOCUMENT = 4u, ATTN_MASK_PREFIX = 8u,
        ATTN_MASK_TEST_QUERY = 16u, ATTN_MASK_GLOBAL = 32u };
 

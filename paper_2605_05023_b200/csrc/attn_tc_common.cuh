@@ -44,10 +44,10 @@ __device__ __forceinline__ void mask_chunk32_bits(uint32_t* y, int a, int e, int
     for (int i = 0; i < 32; ++i)
         if (!(vis & (1u << i))) y[i] = __float_as_uint(-INFINITY);
 }
-__device__ __forceinline__ void mask_chunk32_cmp(uint32_t* y, int a, int e) {
+__device__ __forceinline__ void mask_chunk32_cmp(uint32_t* y, int a, int e, int pre = 0) {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
-        if (i < a || i > e) y[i] = __float_as_uint(-INFINITY);
+        if ((i < a || i > e) && i >= pre) y[i] = __float_as_uint(-INFINITY);
 }
 
 // exp2 of 32 shifted scores -> 16 packed bf16 pairs; accumulates the fp32 row sum in four packed lanes.

@@ -45,7 +45,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kItemWords = 21;                   // {handed over} + the 20 words of a work item, as published in shared memory
+constexpr int kItemWords = 25;                   // {handed over} + the 24 words of a work item, as published in shared memory
 constexpr int kMaxOrdered = 1024;                // query blocks per head that the weight-ordered work list covers
 
 
@@ -105,11 +105,29 @@ struct TileRange {
 struct Item {
     int q0t[2], ht[2]; // per query tile: first query row, query head
     int b, g;          // batch, kv head
+    // Key tiles per query tile, as positions in the item's key-tile list.  Without global tokens the list is the
+    // plain sequence of key tiles (position = tile index).  With global tokens a row sees two pieces, the global
+    // keys [0, global_len) and its own interval, so the item's list is {tiles [0, pend)} followed by {tiles
+    // [pend + jshift, ...)}: position v stands for tile v when v < pend and for tile v + jshift otherwise, both
+    // query tiles walk the whole list (tr[0] = tr[1]; a tile that one of them does not see is masked element-wise
+    // there), and only the producer and the softmax groups, which need the real tile, ever translate.
     TileRange tr[2];
     int lo_max[2], hi_min[2];   // per query tile: keys in [lo_max, hi_min] are visible to every row of the tile
     int doc_first[2], doc_last[2];   // per query tile: documents of its first and last row (first > last: unknown)
     float slope[2];    // per query tile: linear-bias slope of its query head (0 without a slope table)
 };
+// What the instances for masks with global tokens carry in addition.
+struct ItemG : Item {
+    int pend, jshift;
+    int pre_min[2];    // per query tile: keys below pre_min are visible to every row of the tile
+};
+template <bool GLB> using ItemT = std::conditional_t<GLB, ItemG, Item>;
+// Key tile at position pos of an item's key-tile list.
+template <bool GLB, typename I>
+__device__ __forceinline__ int tile_of(const I& it, int pos) {
+    if constexpr (GLB) return pos >= it.pend ? pos + it.jshift : pos;
+    else return pos;
+}
 
 
 // Key tiles that the rows [q0, q0 + 128) can see, and the keys all of them see.
@@ -130,7 +148,7 @@ __device__ __forceinline__ TileRange tile_range(const AttnParams& p, int q0, int
 // `order`, when not null, lists the query blocks of a head heaviest first (packed documents, see build_block_order);
 // otherwise the blocks are taken from the last to the first.
 template <int NQ>
-__device__ __forceinline__ Item decode_item(const AttnParams& p, int lin, const uint16_t* order) {
+__device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const uint16_t* order) {
     // The two query tiles of an item share every K / V tile.  With an even GQA group they are the same 128 rows
     // of two neighbouring query heads of one KV group (identical key ranges: no step in which only one of them
     // has work); otherwise they are 256 consecutive rows of one head (under a causal mask the second tile then
@@ -149,7 +167,7 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin, const 
     const int qb = order ? (int)order[r / sh] : nqb - 1 - r / sh;
     const int bh = sec_start + r % sh;
     const int hq_units = p.Hq / units;
-    Item it;
+    ItemG it;
     it.b = bh / hq_units;
     const int h0 = (bh - it.b * hq_units) * units;
     it.g = h0 / p.group;
@@ -157,13 +175,33 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin, const 
     it.ht[1] = h0 + (pair ? 1 : 0);
     it.q0t[0] = qb * rows;
     it.q0t[1] = qb * rows + (pair ? 0 : kBM);
-    it.tr[0] = tile_range(p, it.q0t[0], it.lo_max[0], it.hi_min[0], it.doc_first[0], it.doc_last[0]);
-    if (pair) {
-        it.tr[1] = it.tr[0];
-        it.lo_max[1] = it.lo_max[0]; it.hi_min[1] = it.hi_min[0];
-        it.doc_first[1] = it.doc_first[0]; it.doc_last[1] = it.doc_last[0];
+    it.pend = 0; it.jshift = 0; it.pre_min[0] = it.pre_min[1] = 0;
+    if (p.mask_flags & kMaskGlobal) {
+        // Union of the two query tiles' key tiles: prefix tiles [0, pend) and window tiles [jlo, jhi).
+        int pend = 0, jlo = 0x7fffffff, jhi = 0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const TileBounds tb = tile_bounds(p, it.q0t[t], kBM);
+            it.lo_max[t] = tb.lo_max; it.hi_min[t] = tb.hi_min; it.doc_first[t] = tb.doc_first; it.doc_last[t] = tb.doc_last;
+            it.pre_min[t] = tb.pre_min;
+            if (!tb.any) continue;
+            pend = max(pend, (tb.pre_max + kBN - 1) / kBN);
+            if (!(tb.hi_max < 0 || tb.lo_min > tb.hi_max)) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
+        }
+        if (jlo >= jhi) { jlo = jhi = pend; }                           // only the global tokens are visible
+        if (jlo <= pend) { jhi = max(jhi, pend); jlo = 0; pend = 0; }   // the two pieces touch: one sequence
+        it.pend = pend;
+        it.jshift = jlo - pend;
+        it.tr[0] = it.tr[1] = TileRange{0, pend + (jhi - jlo)};
     } else {
-        it.tr[1] = tile_range(p, it.q0t[1], it.lo_max[1], it.hi_min[1], it.doc_first[1], it.doc_last[1]);
+        it.tr[0] = tile_range(p, it.q0t[0], it.lo_max[0], it.hi_min[0], it.doc_first[0], it.doc_last[0]);
+        if (pair) {
+            it.tr[1] = it.tr[0];
+            it.lo_max[1] = it.lo_max[0]; it.hi_min[1] = it.hi_min[0];
+            it.doc_first[1] = it.doc_first[0]; it.doc_last[1] = it.doc_last[0];
+        } else {
+            it.tr[1] = tile_range(p, it.q0t[1], it.lo_max[1], it.hi_min[1], it.doc_first[1], it.doc_last[1]);
+        }
     }
     it.slope[0] = p.slopes ? __ldg(p.slopes + it.ht[0]) : 0.f;
     it.slope[1] = p.slopes ? __ldg(p.slopes + it.ht[1]) : 0.f;
@@ -184,7 +222,7 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barr
 template <int NQ>
 __device__ __forceinline__ bool has_block_order(const AttnParams& p) {
     const int rows = p.head_pair ? kBM : NQ * kBM;
-    return (p.mask_flags & kMaskDocument) && (p.Sq + rows - 1) / rows <= kMaxOrdered;
+    return (p.mask_flags & (kMaskDocument | kMaskGlobal)) && (p.Sq + rows - 1) / rows <= kMaxOrdered;
 }
 template <int NQ>
 __device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* order, uint16_t* weight) {   // (its own registers)
@@ -195,9 +233,9 @@ __device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* or
         int jlo = 0x7fffffff, jhi = 0;
         for (int t = 0; t < (p.head_pair ? 1 : NQ); ++t) {
             const TileBounds tb = tile_bounds(p, qb * rows + t * kBM, kBM);
-            if (tb.any) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
+            if (tb.any && tb.hi_max >= 0 && tb.lo_min <= tb.hi_max) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
         }
-        weight[qb] = (uint16_t)min(max(jhi - jlo, 0), 65535);
+        weight[qb] = (uint16_t)min(max(jhi - jlo, 0), 65535);      // (the few tiles of global keys in front are not counted)
     }
     __syncthreads();
     for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
@@ -214,8 +252,8 @@ __device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* or
 // Waits for the next work item published by the scheduler thread, copies it and (kRelease) releases it.  The
 // softmax warps call it with every lane (all lanes need the item) and release once per warp afterwards.
 // Returns false when the grid has no unstarted CTA left (or the wait was abandoned).
-template <bool kRelease = true>
-__device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32_t* status_word, Item& it) {
+template <bool kRelease = true, bool GLB = false>
+__device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32_t* status_word, ItemT<GLB>& it) {
     if (!bounded_wait(ptx::smem_u32(&bars->item_full), phase, bars, status_word)) return false;
     phase ^= 1u;
     const volatile int* m = bars->item_msg;
@@ -225,6 +263,7 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
     it.lo_max[0] = m[9]; it.hi_min[0] = m[10]; it.lo_max[1] = m[11]; it.hi_min[1] = m[12];
     it.doc_first[0] = m[13]; it.doc_last[0] = m[14]; it.doc_first[1] = m[15]; it.doc_last[1] = m[16];
     it.slope[0] = __int_as_float(m[19]); it.slope[1] = __int_as_float(m[20]);
+    if constexpr (GLB) { it.pend = m[21]; it.jshift = m[22]; it.pre_min[0] = m[23]; it.pre_min[1] = m[24]; }
     if constexpr (kRelease) ptx::mbar_arrive(ptx::smem_u32(&bars->item_empty));
     return got != 0;
 }
@@ -246,12 +285,13 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
         volatile int* m = bars->item_msg;
         m[0] = got ? 1 : 0;
         if (got) {
-            const Item it = decode_item<NQ>(p, lin, order);
+            const ItemG it = decode_item<NQ>(p, lin, order);
             m[1] = it.q0t[0]; m[2] = it.q0t[1]; m[3] = it.ht[0]; m[4] = it.ht[1]; m[17] = it.b; m[18] = it.g;
             m[5] = it.tr[0].jlo; m[6] = it.tr[0].jhi; m[7] = it.tr[1].jlo; m[8] = it.tr[1].jhi;
             m[9] = it.lo_max[0]; m[10] = it.hi_min[0]; m[11] = it.lo_max[1]; m[12] = it.hi_min[1];
             m[13] = it.doc_first[0]; m[14] = it.doc_last[0]; m[15] = it.doc_first[1]; m[16] = it.doc_last[1];
             m[19] = __float_as_int(it.slope[0]); m[20] = __float_as_int(it.slope[1]);
+            m[21] = it.pend; m[22] = it.jshift; m[23] = it.pre_min[0]; m[24] = it.pre_min[1];
         }
         ptx::mbar_arrive(ptx::smem_u32(&bars->item_full));
     };
@@ -271,7 +311,7 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
 // ------------------------------------------------------------------------------------------------
 // producer: TMA
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ>
+template <int D, int NQ, bool GLB>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
                                               const CUtensorMap* tmap_v, const AttnParams& p, Barriers* bars,
                                               uint32_t q_smem, uint32_t ring_smem) {
@@ -283,8 +323,9 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
     uint32_t pph = 0, item_phase = 0;
     int q_uses[2] = {0, 0};                         // items in which this Q buffer was loaded so far
 
+    using ItemP = ItemT<GLB>;
     // One K tile: one slot holding D/64 boxes of [128 keys x 64 columns].
-    auto produce_k = [&](const Item& it, int j) -> bool {
+    auto produce_k = [&](const ItemP& it, int j) -> bool {
 #pragma unroll
         for (int sl = 0; sl < C::kSlotsPerTile; ++sl) {
             if (!bounded_wait(ptx::smem_u32(&bars->empty[ps]), pph ^ 1u, bars, p.status_word)) return false;
@@ -293,13 +334,13 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
             ptx::mbar_arrive_expect_tx(bar, C::kSlotBytes);
 #pragma unroll
             for (int bx = 0; bx < C::kSlotBytes / C::kBoxBytes; ++bx)
-                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_k, bar, sl * 128 + bx * 64, j * kBN, it.g, it.b);
+                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_k, bar, sl * 128 + bx * 64, tile_of<GLB>(it, j) * kBN, it.g, it.b);
             if (++ps == C::kStages) { ps = 0; pph ^= 1u; }
         }
         return true;
     };
     // One V tile: one slot of D/64 boxes [128 keys x 64 columns].
-    auto produce_v = [&](const Item& it, int j) -> bool {
+    auto produce_v = [&](const ItemP& it, int j) -> bool {
 #pragma unroll
         for (int sl = 0; sl < C::kSlotsPerTile; ++sl) {
             if (!bounded_wait(ptx::smem_u32(&bars->empty[ps]), pph ^ 1u, bars, p.status_word)) return false;
@@ -308,15 +349,15 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
             ptx::mbar_arrive_expect_tx(bar, C::kSlotBytes);
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx)
-                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_v, bar, bx * 64, j * kBN, it.g, it.b);
+                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_v, bar, bx * 64, tile_of<GLB>(it, j) * kBN, it.g, it.b);
             if (++ps == C::kStages) { ps = 0; pph ^= 1u; }
         }
         return true;
     };
 
     while (true) {
-        Item it;
-        if (!next_item(bars, item_phase, p.status_word, it)) return;
+        ItemP it;
+        if (!next_item<true, GLB>(bars, item_phase, p.status_word, it)) return;
         int J0 = 0x7fffffff, J1 = 0;
 #pragma unroll
         for (int t = 0; t < NQ; ++t) {
@@ -505,7 +546,7 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
 // softmax / sigmoid groups and epilogue: one thread per query row
 // ------------------------------------------------------------------------------------------------
 
-template <int D, int NQ, int SCORE, int NORM>
+template <int D, int NQ, int SCORE, int NORM, bool GLB>
 __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars, uint32_t tmem, int qt) {
     using C = Cfg<D, NQ>;
     constexpr bool SIGMOID = (NORM == kNormSigmoid);   // out_scale * sigmoid(s + b), P as a bf16 hi + lo pair
@@ -523,8 +564,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 
     while (true) {
         // Every lane copies the published item; the warp releases it once all of them have.
-        Item it;
-        const bool got = next_item<false>(bars, item_phase, p.status_word, it);
+        ItemT<GLB> it;
+        const bool got = next_item<false, GLB>(bars, item_phase, p.status_word, it);
         __syncwarp();
         if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->item_empty));
         if (!got) return;
@@ -550,12 +591,15 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         }
 
         for (int n = 0; n < niter; ++n, ++g) {
-            const int kv0 = (tr.jlo + n) * kBN;
+            const int pos = tr.jlo + n;                          // position in the item's key-tile list (see Item)
+            const int kv0 = tile_of<GLB>(it, pos) * kBN;
             const int buf = (NQ == 2) ? qt : (int)(g & 1u);
             const uint32_t ph = (NQ == 2) ? (g & 1u) : ((g >> 1) & 1u);
             // Mask (Appendix A.2): element-wise tests only on tiles that straddle an interval edge.
-            const bool full_tile = (kv0 >= lo_last) && (kv0 + kBN - 1 <= hi_first);
+            bool full_tile = (kv0 >= lo_last) && (kv0 + kBN - 1 <= hi_first);
+            if constexpr (GLB) full_tile = full_tile || (kv0 + kBN - 1 < it.pre_min[qt]);
             const int mask_a = riv.lo - kv0, mask_e = riv.hi - kv0;
+            const int mask_p = GLB ? riv.pre - kv0 : 0;          // global tokens: the columns below it are visible too
             const float rowoff = (float)(ip - kv0);
             if (!bounded_wait(ptx::smem_u32(&bars->s_full[buf]), ph, bars, p.status_word)) return;
             ptx::tc_fence_after_sync();
@@ -599,8 +643,13 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                     if (kMasked) {
                         // One bit test per element (two compares per element made partial tiles cost half as much
                         // again as full ones); the sigmoid and ReLU instances are faster with the compare form.
-                        if constexpr (SIGMOID || RELU) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
-                        else mask_chunk32_bits(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
+                        if constexpr (GLB) {
+                            if constexpr (SIGMOID || RELU) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32, mask_p - c * 32);
+                            else mask_chunk32_bits(&y[c * 32], mask_a - c * 32, mask_e - c * 32, mask_p - c * 32);
+                        } else {
+                            if constexpr (SIGMOID || RELU) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
+                            else mask_chunk32_bits(&y[c * 32], mask_a - c * 32, mask_e - c * 32);
+                        }
                     }
                     if constexpr (!SIGMOID && !RELU) {
     #pragma unroll
@@ -760,7 +809,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 // ------------------------------------------------------------------------------------------------
 // kernel
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ, int SCORE, int NORM>
+template <int D, int NQ, int SCORE, int NORM, bool GLB>      // GLB: masks with global tokens (two key pieces per row)
 __global__ void __launch_bounds__(Cfg<D, NQ>::kThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                    const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnParams p) {
@@ -813,11 +862,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     // NQ = 2: 384 threads x 168 registers at launch; 2 x 128 x 208 + 128 x 88 fits the same budget.
     if (warp < NQ * 4) {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
-        softmax_role<D, NQ, SCORE, NORM>(p, bars, tmem, warp >> 2);
+        softmax_role<D, NQ, SCORE, NORM, GLB>(p, bars, tmem, warp >> 2);
     } else {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         if (warp == C::kProducerWarp) {
-            if (lane == 0) producer_role<D, NQ>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem);
+            if (lane == 0) producer_role<D, NQ, GLB>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem);
         } else if (warp == C::kMmaWarp) {
             if (lane == 0) mma_role<D, NQ, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
@@ -839,10 +888,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ, int SCORE, int NORM>
+template <int D, int NQ, int SCORE, int NORM, bool GLB>
 int launch_instance(AttnParams p, cudaStream_t stream) {
     using C = Cfg<D, NQ>;
-    auto kernel = attn_fwd_tc_kernel<D, NQ, SCORE, NORM>;
+    auto kernel = attn_fwd_tc_kernel<D, NQ, SCORE, NORM, GLB>;
     // The opt-in shared-memory size is a per-device function attribute: set it once per device.
     static SmemAttrFlags attr_set;
     if (!set_smem_attr_once(attr_set, kernel, C::kSmemBytes)) return ATTN_ERR_CUDA;
@@ -872,13 +921,18 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
+template <int D, int NQ, bool GLB>
+int launch_for_mask(const AttnParams& p, cudaStream_t stream) {
+    if (p.normalizer == kNormSigmoid) return launch_instance<D, NQ, kScoreGeneric, kNormSigmoid, GLB>(p, stream);
+    if (p.normalizer == kNormRelu) return launch_instance<D, NQ, kScoreGeneric, kNormRelu, GLB>(p, stream);
+    if (p.softcap > 0.f) return launch_instance<D, NQ, kScoreGeneric, kNormSoftmax, GLB>(p, stream);
+    if (p.slopes) return launch_instance<D, NQ, kScoreBias, kNormSoftmax, GLB>(p, stream);
+    return launch_instance<D, NQ, kScorePlain, kNormSoftmax, GLB>(p, stream);
+}
+// Masks with global tokens get their own instances, so that the others carry none of the two-piece walk.
 template <int D, int NQ>
 int launch_for_d(const AttnParams& p, cudaStream_t stream) {
-    if (p.normalizer == kNormSigmoid) return launch_instance<D, NQ, kScoreGeneric, kNormSigmoid>(p, stream);
-    if (p.normalizer == kNormRelu) return launch_instance<D, NQ, kScoreGeneric, kNormRelu>(p, stream);
-    if (p.softcap > 0.f) return launch_instance<D, NQ, kScoreGeneric, kNormSoftmax>(p, stream);
-    if (p.slopes) return launch_instance<D, NQ, kScoreBias, kNormSoftmax>(p, stream);
-    return launch_instance<D, NQ, kScorePlain, kNormSoftmax>(p, stream);
+    return (p.mask_flags & kMaskGlobal) ? launch_for_mask<D, NQ, true>(p, stream) : launch_for_mask<D, NQ, false>(p, stream);
 }
 
 }  // namespace
@@ -897,9 +951,10 @@ int launch_attn_fwd_bf16(const AttnParams& p, cudaStream_t stream, int* launches
     static const bool force_split = []() { const char* e = getenv("B200ATTN_FORCE_SPLIT"); return e && e[0] == '1'; }();
     static const bool force_pair = []() { const char* e = getenv("B200ATTN_FORCE_PAIR"); return e && e[0] == '1'; }();
     int rc;
-    if (force_split || (p.mask_flags & kMaskGlobal)) {      // two key intervals per row: only the one-tile kernel walks them
+    const bool global = (p.mask_flags & kMaskGlobal) != 0;
+    if (force_split || (global && (p.D == 256 || force_pair))) {   // two key pieces per row: not on the CTA-pair kernel
         rc = launch_attn_fwd_bf16_split(p, stream);
-    } else if (p.D == 256 || (p.D == 128 && (force_pair || p.normalizer == kNormSigmoid))) {
+    } else if (p.D == 256 || (p.D == 128 && !global && (force_pair || p.normalizer == kNormSigmoid))) {
         rc = launch_attn_fwd_bf16_pair(p, stream);
     } else {
         switch (p.D) {
