@@ -76,64 +76,90 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML from a background thread.  The thread is started ahead
+    of the timed region (its first queries are slow) and keeps sampling; ``begin()`` / ``end()`` mark the region,
+    and the summary covers the samples taken between the two marks."""
 
     def __init__(self, index: int, period_s: float = 0.002):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.max_mhz = [], None          # (time, MHz, reason mask)
         self.period_s = period_s
         self._stop = threading.Event()
         self._thread = None
+        self._t0 = self._t1 = None
         try:
             import pynvml
             pynvml.nvmlInit()
             self._nv = pynvml
             self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
-            # The first NVML queries on a fresh process can take long and contend with kernel launches:
-            # make them here, before anything is timed.
             pynvml.nvmlDeviceGetClockInfo(self._h, pynvml.NVML_CLOCK_SM)
         except Exception:
             self._nv = None
 
-    def _run(self):
+    def _reason_names(self):
         nv = self._nv
-        names = {
+        return {
             getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
             getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
             getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
             getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
             getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
         }
+
+    def _run(self):
+        nv = self._nv
         while not self._stop.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
                 try:
                     mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
                 except Exception:
                     mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
-                for bit, name in names.items():
-                    if mask & bit:
-                        self.reasons.add(name)
+                self.samples.append((time.perf_counter(), mhz, mask))
             except Exception:
                 pass
             time.sleep(self.period_s)
 
-    def __enter__(self):
-        if self._nv is not None:
+    def start(self):
+        if self._nv is not None and self._thread is None:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
+            time.sleep(0.02)                    # let the first (slow) queries pass before anything is timed
         return self
 
-    def __exit__(self, *exc):
+    def begin(self):
+        self._t0 = time.perf_counter()
+
+    def end(self):
+        self._t1 = time.perf_counter()
+
+    def stop(self):
         self._stop.set()
         if self._thread is not None:
             self._thread.join()
 
+    # context-manager form: the whole block is the region
+    def __enter__(self):
+        self.start()
+        self.begin()
+        return self
+
+    def __exit__(self, *exc):
+        self.end()
+        self.stop()
+
     def summary(self):
-        if not self.samples:
-            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
-        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        t0 = self._t0 if self._t0 is not None else 0.0
+        t1 = self._t1 if self._t1 is not None else float("inf")
+        inside = [(m, r) for t, m, r in self.samples if t0 <= t <= t1]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        mask = 0
+        for _, r in inside:
+            mask |= r
+        reasons = sorted(name for bit, name in self._reason_names().items() if mask & bit)
+        return {"sm_mhz": float(np.median([m for m, _ in inside])), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(inside)}
 
 
 def physical_gpu_index(local: int) -> int:
@@ -160,6 +186,11 @@ def config_block(workload_key, workloads):
             "per_rank": "same workload on every GPU, different seeds, no collective"}, flushed
 
 
+# Multiply-adds (rows x keys x head dimension, summed over the step's variants) of one oracle sample: about 20 s on
+# the 16 host cores of this pool's GPU machines.
+ORACLE_SAMPLE_WORK = 2.0e11
+
+
 def oracle_sample(workloads, target_rows):
     """Times the float64 oracle, as it stands, on evenly spaced rows of each variant.
     Returns (TFLOP/s over the unmasked FLOPs of those rows, threads, description, seconds)."""
@@ -176,7 +207,8 @@ def oracle_sample(workloads, target_rows):
                             out_scale=w.out_scale, cu_seqlens=w.cu_seqlens, prefix_len=w.prefix_len,
                             test_query_start=w.test_query_start, global_len=w.global_len)
         total = w.B * w.Hq * w.Sq
-        n = min(total, target_rows)
+        # the oracle computes every score of a row (all Sk keys): bound the sample's work, not only its row count
+        n = max(64, min(total, target_rows, int(ORACLE_SAMPLE_WORK / (w.Sk * w.D * len(workloads)))))
         rows = np.unique(np.linspace(0, total - 1, n).astype(np.int64))
         oracle.attn_fwd_rows(q, k, v, var, rows[:8])            # page the library and inputs in
         t0 = time.perf_counter()
@@ -558,12 +590,16 @@ def run_attention(args, rank, world, local):
         kernel_events = []
         t_start = torch.cuda.Event(enable_timing=True)
         t_stop = torch.cuda.Event(enable_timing=True)
-        with ClockSampler(gpu_index, period_s=0.001) as clocks:
-            t_start.record(stream)
-            for _ in range(args.steps):
-                step(kernel_events)
-            t_stop.record(stream)
-            barrier()
+        clocks = ClockSampler(gpu_index, period_s=0.0005).start()
+        barrier()
+        clocks.begin()
+        t_start.record(stream)
+        for _ in range(args.steps):
+            step(kernel_events)
+        t_stop.record(stream)
+        barrier()
+        clocks.end()
+        clocks.stop()
         launches = pk.launch_count() - launches0
         bad = status_error(cases)
         if world > 1:   # every rank repeats if any rank has to
