@@ -33,7 +33,8 @@ std::atomic<long long> g_map_hits{0};
 
 bool same_key(const MapKey& a, const MapKey& b) {
     return a.ptr == b.ptr && a.B == b.B && a.H == b.H && a.S == b.S && a.D == b.D && a.st[0] == b.st[0] &&
-           a.st[1] == b.st[1] && a.st[2] == b.st[2] && a.box_rows == b.box_rows && a.box_cols == b.box_cols;
+           a.st[1] == b.st[1] && a.st[2] == b.st[2] && a.box_rows == b.box_rows && a.box_cols == b.box_cols &&
+           a.swizzle_bytes == b.swizzle_bytes;
 }
 size_t slot_of(const MapKey& k) {
     uint64_t h = reinterpret_cast<uintptr_t>(k.ptr) * 0x9E3779B97F4A7C15ull;

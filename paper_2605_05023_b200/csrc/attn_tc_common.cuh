@@ -114,6 +114,7 @@ struct MapKey {
     int B, H, S, D;
     long long st[3];
     int box_rows, box_cols;
+    int swizzle_bytes;      // 128 (operand tiles) or 64 (32-column output boxes)
 };
 inline bool encode_map(CUtensorMap* map, const MapKey& k) {
     EncodeTiledFn fn = encode_fn();
@@ -123,7 +124,8 @@ inline bool encode_map(CUtensorMap* map, const MapKey& k) {
     const cuuint32_t box[4] = {(cuuint32_t)k.box_cols, (cuuint32_t)k.box_rows, 1u, 1u};
     const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k.ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, k.swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 // Encoded maps are cached by key (attn_api.cu; emptied by attn_clear_cache()).
@@ -132,8 +134,8 @@ void clear_map_cache();
 long long map_cache_hits();
 
 inline bool make_map(CUtensorMap* map, const void* ptr, int B, int H, int S, int D, const long long st[3], int box_rows,
-                     int box_cols = 64) {
-    const MapKey key = {ptr, B, H, S, D, {st[0], st[1], st[2]}, box_rows, box_cols};
+                     int box_cols = 64, int swizzle_bytes = 128) {
+    const MapKey key = {ptr, B, H, S, D, {st[0], st[1], st[2]}, box_rows, box_cols, swizzle_bytes};
     return cached_map(map, key);
 }
 

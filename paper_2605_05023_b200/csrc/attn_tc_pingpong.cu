@@ -46,10 +46,9 @@ namespace {
 using namespace tc;
 
 constexpr int kItemWords = 25;                   // {handed over} + the 24 words of a work item, as published in shared memory
-constexpr int kMaxOrdered = 1024;                // query blocks per head that the weight-ordered work list covers
 
 
-template <int D, int NQ>
+template <int D, int NQ, bool TMA_OUT = false>
 struct Cfg {
     static constexpr int kBoxBytes = 64 * 128 * 2;                      // one 64-column TMA box of 128 rows
     static constexpr int kSlotBytes = (D == 64) ? kBoxBytes : 2 * kBoxBytes;
@@ -58,8 +57,12 @@ struct Cfg {
     static constexpr int kQBytes = kBM * D * 2;
     static constexpr int kDataBytes = NQ * kQBytes + kStages * kSlotBytes;
     static constexpr int kBarBytes = 1024;
+    static constexpr int kMaxOrdered = TMA_OUT ? 256 : 1024;            // query blocks per head that the weight-ordered work list covers
     static constexpr int kOrderBytes = 2 * kMaxOrdered * 2;             // query-block order and weights (packed documents)
-    static constexpr int kSmemBytes = kDataBytes + kBarBytes + kOrderBytes + 1024;    // + slack to align the base to 1024
+    static constexpr int kStageBytes = 32 * 32 * 2;                     // a 32-row x 32-column bf16 box of O
+    static constexpr int kOutBytes = TMA_OUT ? NQ * 4 * 2 * kStageBytes : 0;   // two such boxes per softmax warp
+    static constexpr int kSmemBytes = kDataBytes + kOutBytes + kBarBytes + kOrderBytes + 1024;    // + slack to align the base to 1024
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
     // Softmax warpgroups first, then one warpgroup holding the producer, MMA and scheduler warps.
     // With NQ = 2 setmaxnreg moves registers from that last warpgroup to the softmax groups.
     static constexpr int kThreads = NQ * 128 + 128;
@@ -218,17 +221,17 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, Barr
 // blocks once, in shared memory, before its roles start: weight = key tiles of the block's work item; rank =
 // blocks that are heavier, plus equally heavy blocks of lower index (a stable counting of all pairs, spread over
 // the CTA's threads, with no atomics, so that all CTAs agree on the order).  The order is used when the mask has a
-// document clause and there are at most kMaxOrdered blocks.
+// document (or global-token) clause and the blocks fit the table.
 template <int NQ>
-__device__ __forceinline__ bool has_block_order(const AttnParams& p) {
+__device__ __forceinline__ bool has_block_order(const AttnParams& p, int capacity) {
     const int rows = p.head_pair ? kBM : NQ * kBM;
-    return (p.mask_flags & (kMaskDocument | kMaskGlobal)) && (p.Sq + rows - 1) / rows <= kMaxOrdered;
+    return (p.mask_flags & (kMaskDocument | kMaskGlobal)) && (p.Sq + rows - 1) / rows <= capacity;
 }
 template <int NQ>
-__device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* order, uint16_t* weight) {   // (its own registers)
+__device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* order, uint16_t* weight, int capacity) {   // (its own registers)
     const int rows = p.head_pair ? kBM : NQ * kBM;
     const int nqb = (p.Sq + rows - 1) / rows;
-    if (!has_block_order<NQ>(p)) return;
+    if (!has_block_order<NQ>(p, capacity)) return;
     for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
         int jlo = 0x7fffffff, jhi = 0;
         for (int t = 0; t < (p.head_pair ? 1 : NQ); ++t) {
@@ -276,9 +279,9 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
 // only this thread touches the hardware scheduler's response).  It publishes {handed over, decoded item} with
 // ordinary stores for the other roles, so that no role spends time on index arithmetic and mask intervals.
 template <int NQ>
-__device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* bars) {
+__device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* bars, int order_capacity) {
     // the heaviest-first order of the query blocks sits right behind the barrier block (see build_block_order)
-    const uint16_t* order = has_block_order<NQ>(p) ? reinterpret_cast<const uint16_t*>(reinterpret_cast<const uint8_t*>(bars) + 1024) : nullptr;
+    const uint16_t* order = has_block_order<NQ>(p, order_capacity) ? reinterpret_cast<const uint16_t*>(reinterpret_cast<const uint8_t*>(bars) + 1024) : nullptr;
     int32_t* status_word = p.status_word;
     uint32_t clc_phase = 0, empty_phase = 0;
     auto publish = [&](bool got, int lin) {
@@ -546,9 +549,10 @@ __device__ __forceinline__ void mma_role(const AttnParams& p, Barriers* bars, ui
 // softmax / sigmoid groups and epilogue: one thread per query row
 // ------------------------------------------------------------------------------------------------
 
-template <int D, int NQ, int SCORE, int NORM, bool GLB>
-__device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars, uint32_t tmem, int qt) {
-    using C = Cfg<D, NQ>;
+template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
+__device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars, uint32_t tmem, int qt, const CUtensorMap* tmap_o,
+                                             uint32_t stage_smem, uint8_t* stage_ptr) {
+    using C = Cfg<D, NQ, TMA_OUT>;
     constexpr bool SIGMOID = (NORM == kNormSigmoid);   // out_scale * sigmoid(s + b), P as a bf16 hi + lo pair
     constexpr bool RELU = (NORM == kNormRelu);         // out_scale * max(s, 0), no exponential at all
     const int wg_thread = threadIdx.x & 127;                 // row within the tile
@@ -780,14 +784,18 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 #pragma unroll
                 for (int i = 0; i < 32; ++i) orr[i] = 0u;
             }
-            if (store_row) {
-                if (p.o_fp32) {
+            if (p.o_fp32) {
+                if (store_row) {
                     float4* dst = reinterpret_cast<float4*>(obase + c * 128);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         dst[i] = make_float4(__uint_as_float(orr[4 * i]) * inv, __uint_as_float(orr[4 * i + 1]) * inv,
                                              __uint_as_float(orr[4 * i + 2]) * inv, __uint_as_float(orr[4 * i + 3]) * inv);
-                } else {
+                }
+            } else if constexpr (!TMA_OUT) {
+                // bf16 output, 256 consecutive rows per item: the first tile's epilogue runs under the second tile's
+                // last key step and the threads go on at once, so plain 16-byte stores by the row's owner are best.
+                if (store_row) {
                     uint4* dst = reinterpret_cast<uint4*>(obase + c * 64);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -799,6 +807,32 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         dst[i] = w;
                     }
                 }
+            } else {
+                // bf16 output, two heads x 128 rows per item (both tiles end together and their epilogues compete
+                // for the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
+                // in shared memory (64-byte swizzle: the 16-byte piece k of row r sits at piece k ^ ((r >> 1) & 3),
+                // conflict free) and leave as one TMA tile store, which also clips rows beyond Sq.  A thread-owns-a-row
+                // store to global memory touches 32 lines per instruction; this way the stores cost the load/store
+                // unit an eighth of that.
+                const int r = threadIdx.x & 31;
+                if (r == 0) ptx::bulk_wait_group_read1();        // the store before last has been read out of its box
+                __syncwarp();
+                uint4* dst = reinterpret_cast<uint4*>(stage_ptr + (c & 1) * C::kStageBytes + r * 64);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 w;
+                    w.x = ptx::pack_bf16x2(__uint_as_float(orr[8 * i]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
+                    w.y = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
+                    w.z = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
+                    w.w = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
+                    dst[i ^ ((r >> 1) & 3)] = w;
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (r == 0) {
+                    ptx::tma_store_4d(tmap_o, stage_smem + (c & 1) * C::kStageBytes, c * 32, q0 + (wg_thread & ~31), it.ht[qt], it.b);
+                    ptx::bulk_commit_group();
+                }
             }
         }
         if (!SIGMOID && !RELU && p.lse && store_row)
@@ -809,18 +843,21 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 // ------------------------------------------------------------------------------------------------
 // kernel
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ, int SCORE, int NORM, bool GLB>      // GLB: masks with global tokens (two key pieces per row)
+// GLB: masks with global tokens (two key pieces per row).  TMA_OUT: bf16 output through shared memory and TMA tile
+// stores (work items of two heads x 128 rows).
+template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
 __global__ void __launch_bounds__(Cfg<D, NQ>::kThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                   const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnParams p) {
-    using C = Cfg<D, NQ>;
+                   const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                   const __grid_constant__ AttnParams p) {
+    using C = Cfg<D, NQ, TMA_OUT>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     const uint32_t q_smem = base;
     const uint32_t ring_smem = base + NQ * C::kQBytes;
-    Barriers* bars = reinterpret_cast<Barriers*>(smem + C::kDataBytes);
+    Barriers* bars = reinterpret_cast<Barriers*>(smem + C::kDataBytes + C::kOutBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -851,8 +888,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     }
     static_assert(C::kBarBytes == 1024, "scheduler_role finds the block order 1024 bytes behind the barriers");
     {
-        uint16_t* order = reinterpret_cast<uint16_t*>(smem + C::kDataBytes + C::kBarBytes);
-        build_block_order<NQ>(p, order, order + kMaxOrdered);
+        uint16_t* order = reinterpret_cast<uint16_t*>(smem + C::kDataBytes + C::kOutBytes + C::kBarBytes);
+        build_block_order<NQ>(p, order, order + C::kMaxOrdered, C::kMaxOrdered);
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -862,7 +899,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     // NQ = 2: 384 threads x 168 registers at launch; 2 x 128 x 208 + 128 x 88 fits the same budget.
     if (warp < NQ * 4) {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(C::kRegsSoftmax));
-        softmax_role<D, NQ, SCORE, NORM, GLB>(p, bars, tmem, warp >> 2);
+        softmax_role<D, NQ, SCORE, NORM, GLB, TMA_OUT>(p, bars, tmem, warp >> 2, &tmap_o, base + C::kDataBytes + warp * 2 * C::kStageBytes,
+                                              smem + C::kDataBytes + warp * 2 * C::kStageBytes);
+        if (TMA_OUT && lane == 0) ptx::bulk_wait_group0();          // this warp's output boxes have left shared memory
     } else {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         if (warp == C::kProducerWarp) {
@@ -870,7 +909,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         } else if (warp == C::kMmaWarp) {
             if (lane == 0) mma_role<D, NQ, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
-            if (lane == 0) scheduler_role<NQ>(p, bars);
+            if (lane == 0) scheduler_role<NQ>(p, bars, C::kMaxOrdered);
         } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
             check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
@@ -888,17 +927,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ, int SCORE, int NORM, bool GLB>
+template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
 int launch_instance(AttnParams p, cudaStream_t stream) {
-    using C = Cfg<D, NQ>;
-    auto kernel = attn_fwd_tc_kernel<D, NQ, SCORE, NORM, GLB>;
+    using C = Cfg<D, NQ, TMA_OUT>;
+    auto kernel = attn_fwd_tc_kernel<D, NQ, SCORE, NORM, GLB, TMA_OUT>;
     // The opt-in shared-memory size is a per-device function attribute: set it once per device.
     static SmemAttrFlags attr_set;
     if (!set_smem_attr_once(attr_set, kernel, C::kSmemBytes)) return ATTN_ERR_CUDA;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     if (!make_map(&mq, p.q, p.B, p.Hq, p.Sq, D, p.qs, 128) || !make_map(&mk, p.k, p.B, p.Hkv, p.Sk, D, p.ks, 128) ||
         !make_map(&mv, p.v, p.B, p.Hkv, p.Sk, D, p.vs, 128))
         return ATTN_ERR_CUDA;
+    // TMA_OUT instances store bf16 output as tiles of 32 rows x 32 columns; the others get a placeholder map that
+    // they never use.
+    if (!TMA_OUT) mo = mq;
+    else if (!make_map(&mo, p.o, p.B, p.Hq, p.Sq, D, p.os, 32, 32, 64)) return ATTN_ERR_CUDA;
     // Heads per section of the work order: as many KV heads as keep the section's K and V within
     // about 40 MB of L2, in equal sections, whole GQA groups.
     const long long kv_bytes = 2ll * p.Sk * D * 2;
@@ -917,22 +960,25 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     const long long nqb = (p.Sq + rows - 1) / rows;
     const long long grid = nqb * (bh / (p.head_pair ? 2 : 1));
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
-    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, p);
+    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
 
-template <int D, int NQ, bool GLB>
+template <int D, int NQ, bool GLB, bool TMA_OUT>
 int launch_for_mask(const AttnParams& p, cudaStream_t stream) {
-    if (p.normalizer == kNormSigmoid) return launch_instance<D, NQ, kScoreGeneric, kNormSigmoid, GLB>(p, stream);
-    if (p.normalizer == kNormRelu) return launch_instance<D, NQ, kScoreGeneric, kNormRelu, GLB>(p, stream);
-    if (p.softcap > 0.f) return launch_instance<D, NQ, kScoreGeneric, kNormSoftmax, GLB>(p, stream);
-    if (p.slopes) return launch_instance<D, NQ, kScoreBias, kNormSoftmax, GLB>(p, stream);
-    return launch_instance<D, NQ, kScorePlain, kNormSoftmax, GLB>(p, stream);
+    if (p.normalizer == kNormSigmoid) return launch_instance<D, NQ, kScoreGeneric, kNormSigmoid, GLB, TMA_OUT>(p, stream);
+    if (p.normalizer == kNormRelu) return launch_instance<D, NQ, kScoreGeneric, kNormRelu, GLB, TMA_OUT>(p, stream);
+    if (p.softcap > 0.f) return launch_instance<D, NQ, kScoreGeneric, kNormSoftmax, GLB, TMA_OUT>(p, stream);
+    if (p.slopes) return launch_instance<D, NQ, kScoreBias, kNormSoftmax, GLB, TMA_OUT>(p, stream);
+    return launch_instance<D, NQ, kScorePlain, kNormSoftmax, GLB, TMA_OUT>(p, stream);
 }
-// Masks with global tokens get their own instances, so that the others carry none of the two-piece walk.
+// Masks with global tokens get their own instances, so that the others carry none of the two-piece walk; work items
+// of two heads x 128 rows (even GQA group) with bf16 output get the instances whose epilogue goes through TMA stores.
 template <int D, int NQ>
 int launch_for_d(const AttnParams& p, cudaStream_t stream) {
-    return (p.mask_flags & kMaskGlobal) ? launch_for_mask<D, NQ, true>(p, stream) : launch_for_mask<D, NQ, false>(p, stream);
+    if (p.mask_flags & kMaskGlobal) return launch_for_mask<D, NQ, true, false>(p, stream);
+    if (p.group % 2 == 0 && !p.o_fp32) return launch_for_mask<D, NQ, false, true>(p, stream);
+    return launch_for_mask<D, NQ, false, false>(p, stream);
 }
 
 }  // namespace
