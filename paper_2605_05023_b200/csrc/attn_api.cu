@@ -1,6 +1,6 @@
 // Host side of the C ABI declared in include/attn.h: argument validation, parameter block, kernel selection,
 // and the cache of encoded TMA tensor maps.  Nothing here computes; every step of the path runs in the kernels
-// of attn_simt_fp32.cu (fp32 inputs) and attn_tc_pingpong.cu / attn_tc_pair.cu / attn_tc_split.cu (bf16 inputs,
+// of attn_simt_fp32.cu (fp32 inputs) and attn_tc_pingpong*.cu / attn_tc_pair.cu / attn_tc_split.cu (bf16 inputs,
 // tcgen05).
 #include <atomic>
 #include <cmath>

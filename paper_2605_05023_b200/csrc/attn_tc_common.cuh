@@ -1,4 +1,4 @@
-// Pieces shared by the three tensor-core attention kernels (attn_tc_pingpong.cu, attn_tc_pair.cu,
+// Pieces shared by the three tensor-core attention kernels (attn_tc_pingpong.cuh, attn_tc_pair.cu,
 // attn_tc_split.cu): tile sizes and constants, the tcgen05 instruction descriptor, the element-wise mask of a
 // partial tile, the exponential step of the online softmax, and the host-side TMA tensor maps.  (Bounded waits,
 // the work-item fetch and the warp-level arrivals are in sm100_sync.cuh.)

@@ -748,7 +748,7 @@ int launch_for_d(const AttnParams& p, cudaStream_t stream) {
 
 // One query tile per work item, S double buffered, two column-split softmax groups: the kernel for D = 256
 // (its accumulator leaves no TMEM room for a second query tile).  It is also correct for D = 64 and 128, where
-// the two-tile kernel of attn_tc_pingpong.cu is faster because it reads K and V from L2 half as often.
+// the two-tile kernel of attn_tc_pingpong.cuh is faster because it reads K and V from L2 half as often.
 int launch_attn_fwd_bf16_split(const AttnParams& p, cudaStream_t stream) {
     switch (p.D) {
         case 64: return launch_for_d<64>(p, stream);
