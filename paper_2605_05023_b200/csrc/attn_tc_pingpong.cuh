@@ -46,7 +46,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kItemWords = 25;                   // {handed over} + the 24 words of a work item, as published in shared memory
+constexpr int kItemWords = 26;                   // {handed over} + the 25 words of a work item, as published in shared memory
 
 
 template <int D, int NQ, bool TMA_OUT = false>
@@ -119,6 +119,11 @@ struct Item {
     int lo_max[2], hi_min[2];   // per query tile: keys in [lo_max, hi_min] are visible to every row of the tile
     int doc_first[2], doc_last[2];   // per query tile: documents of its first and last row (first > last: unknown)
     float slope[2];    // per query tile: linear-bias slope of its query head (0 without a slope table)
+    // Key tiles are walked downwards, from the last one to the first, when rev_top >= 0: position v of the list then
+    // stands for tile rev_top - v and tr[] holds positions.  The scheduler asks for it when the heads' position bias
+    // has a negative slope (ALiBi): the bias, and with it the row maximum, then falls from tile to tile instead of
+    // growing by slope * 128 per tile, which at the steeper slopes forced a rescaling of O at every key step.
+    int rev_top;
 };
 // What the instances for masks with global tokens carry in addition.
 struct ItemG : Item {
@@ -126,10 +131,11 @@ struct ItemG : Item {
     int pre_min[2];    // per query tile: keys below pre_min are visible to every row of the tile
 };
 template <bool GLB> using ItemT = std::conditional_t<GLB, ItemG, Item>;
-// Key tile at position pos of an item's key-tile list.
-template <bool GLB, typename I>
+// Key tile at position pos of an item's key-tile list.  REV: instances whose scheduler may reverse the walk.
+template <bool GLB, bool REV, typename I>
 __device__ __forceinline__ int tile_of(const I& it, int pos) {
     if constexpr (GLB) return pos >= it.pend ? pos + it.jshift : pos;
+    else if constexpr (REV) return it.rev_top >= 0 ? it.rev_top - pos : pos;
     else return pos;
 }
 
@@ -209,6 +215,19 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     }
     it.slope[0] = p.slopes ? __ldg(p.slopes + it.ht[0]) : 0.f;
     it.slope[1] = p.slopes ? __ldg(p.slopes + it.ht[1]) : 0.f;
+    it.rev_top = -1;
+    if (!(p.mask_flags & kMaskGlobal) && (it.slope[0] < 0.f || it.slope[1] < 0.f)) {
+        // walk the key tiles downwards: tile j becomes position (top - j)
+        int top = 0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) top = max(top, it.tr[t].jhi);
+        if (top > 0) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+                it.tr[t] = (it.tr[t].jlo < it.tr[t].jhi) ? TileRange{top - it.tr[t].jhi, top - it.tr[t].jlo} : TileRange{0, 0};
+            it.rev_top = top - 1;
+        }
+    }
     return it;
 }
 
@@ -256,7 +275,7 @@ __device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* or
 // Waits for the next work item published by the scheduler thread, copies it and (kRelease) releases it.  The
 // softmax warps call it with every lane (all lanes need the item) and release once per warp afterwards.
 // Returns false when the grid has no unstarted CTA left (or the wait was abandoned).
-template <bool kRelease = true, bool GLB = false>
+template <bool kRelease = true, bool GLB = false, bool REV = false>
 __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32_t* status_word, ItemT<GLB>& it) {
     if (!bounded_wait(ptx::smem_u32(&bars->item_full), phase, bars, status_word)) return false;
     phase ^= 1u;
@@ -268,6 +287,7 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
     it.doc_first[0] = m[13]; it.doc_last[0] = m[14]; it.doc_first[1] = m[15]; it.doc_last[1] = m[16];
     it.slope[0] = __int_as_float(m[19]); it.slope[1] = __int_as_float(m[20]);
     if constexpr (GLB) { it.pend = m[21]; it.jshift = m[22]; it.pre_min[0] = m[23]; it.pre_min[1] = m[24]; }
+    if constexpr (REV) it.rev_top = m[25];
     if constexpr (kRelease) ptx::mbar_arrive(ptx::smem_u32(&bars->item_empty));
     return got != 0;
 }
@@ -296,6 +316,7 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
             m[13] = it.doc_first[0]; m[14] = it.doc_last[0]; m[15] = it.doc_first[1]; m[16] = it.doc_last[1];
             m[19] = __float_as_int(it.slope[0]); m[20] = __float_as_int(it.slope[1]);
             m[21] = it.pend; m[22] = it.jshift; m[23] = it.pre_min[0]; m[24] = it.pre_min[1];
+            m[25] = it.rev_top;
         }
         ptx::mbar_arrive(ptx::smem_u32(&bars->item_full));
     };
@@ -315,7 +336,7 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
 // ------------------------------------------------------------------------------------------------
 // producer: TMA
 // ------------------------------------------------------------------------------------------------
-template <int D, int NQ, bool GLB>
+template <int D, int NQ, bool GLB, bool REV>
 __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const CUtensorMap* tmap_k,
                                               const CUtensorMap* tmap_v, const AttnParams& p, Barriers* bars,
                                               uint32_t q_smem, uint32_t ring_smem) {
@@ -338,7 +359,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
             ptx::mbar_arrive_expect_tx(bar, C::kSlotBytes);
 #pragma unroll
             for (int bx = 0; bx < C::kSlotBytes / C::kBoxBytes; ++bx)
-                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_k, bar, sl * 128 + bx * 64, tile_of<GLB>(it, j) * kBN, it.g, it.b);
+                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_k, bar, sl * 128 + bx * 64, tile_of<GLB, REV>(it, j) * kBN, it.g, it.b);
             if (++ps == C::kStages) { ps = 0; pph ^= 1u; }
         }
         return true;
@@ -353,7 +374,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
             ptx::mbar_arrive_expect_tx(bar, C::kSlotBytes);
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx)
-                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_v, bar, bx * 64, tile_of<GLB>(it, j) * kBN, it.g, it.b);
+                ptx::tma_load_4d(dst + bx * C::kBoxBytes, tmap_v, bar, bx * 64, tile_of<GLB, REV>(it, j) * kBN, it.g, it.b);
             if (++ps == C::kStages) { ps = 0; pph ^= 1u; }
         }
         return true;
@@ -361,7 +382,7 @@ __device__ __forceinline__ void producer_role(const CUtensorMap* tmap_q, const C
 
     while (true) {
         ItemP it;
-        if (!next_item<true, GLB>(bars, item_phase, p.status_word, it)) return;
+        if (!next_item<true, GLB, REV>(bars, item_phase, p.status_word, it)) return;
         int J0 = 0x7fffffff, J1 = 0;
 #pragma unroll
         for (int t = 0; t < NQ; ++t) {
@@ -570,7 +591,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
     while (true) {
         // Every lane copies the published item; the warp releases it once all of them have.
         ItemT<GLB> it;
-        const bool got = next_item<false, GLB>(bars, item_phase, p.status_word, it);
+        const bool got = next_item<false, GLB, SCORE != kScorePlain>(bars, item_phase, p.status_word, it);
         __syncwarp();
         if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->item_empty));
         if (!got) return;
@@ -597,7 +618,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 
         for (int n = 0; n < niter; ++n, ++g) {
             const int pos = tr.jlo + n;                          // position in the item's key-tile list (see Item)
-            const int kv0 = tile_of<GLB>(it, pos) * kBN;
+            const int kv0 = tile_of<GLB, SCORE != kScorePlain>(it, pos) * kBN;
             const int buf = (NQ == 2) ? qt : (int)(g & 1u);
             const uint32_t ph = (NQ == 2) ? (g & 1u) : ((g >> 1) & 1u);
             // Mask (Appendix A.2): element-wise tests only on tiles that straddle an interval edge.
@@ -906,7 +927,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
     } else {
         if constexpr (NQ == 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(C::kRegsOther));
         if (warp == C::kProducerWarp) {
-            if (lane == 0) producer_role<D, NQ, GLB>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem);
+            if (lane == 0) producer_role<D, NQ, GLB, SCORE != kScorePlain>(&tmap_q, &tmap_k, &tmap_v, p, bars, q_smem, ring_smem);
         } else if (warp == C::kMmaWarp) {
             if (lane == 0) mma_role<D, NQ, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
