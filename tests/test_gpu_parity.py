@@ -177,6 +177,16 @@ BF16_EXTRA = [
              cu_seqlens=(0, 300, 301, 512, 640, 1000, 1024), global_len=300),
     Workload("b_share_question_sigmoid", 1, 1, 1, 640, 640, 128, seed=70, causal=True, cu_seqlens=(0, 128, 384, 640),
              global_len=128, normalizer="sigmoid", o_dtype="fp32", sigmoid_bias=-math.log(640.0), std=1.5),
+    # key tiles walked downwards (negative slopes): both heads of an item, one of them only, with documents, with an
+    # odd GQA group (256-row items: the second tile starts alone), Sq < Sk, and a non-causal two-sided window
+    Workload("b_alibi_pair_mixed", 1, 4, 2, 700, 700, 128, seed=130, causal=True, slopes=(-0.5, 0.25, 0.0, -0.01)),
+    Workload("b_alibi_docs", 1, 4, 2, 1024, 1024, 128, seed=131, causal=True, slopes=alibi_slopes(4),
+             cu_seqlens=(0, 130, 131, 500, 1024)),
+    Workload("b_alibi_odd_group", 1, 3, 1, 900, 900, 128, seed=132, causal=True, slopes=(-0.3, -0.02, -1.0)),
+    Workload("b_alibi_sq_lt_sk", 1, 2, 1, 300, 800, 64, seed=133, causal=True, window_left=400, window_right=0,
+             slopes=(-0.1, -0.7)),
+    Workload("b_alibi_two_sided", 1, 2, 2, 700, 700, 128, seed=134, window_left=200, window_right=150, slopes=(-0.05, -0.2)),
+    Workload("b_alibi_softcap", 1, 2, 2, 640, 640, 128, seed=135, causal=True, softcap=30.0, slopes=(-0.4, -0.02), std=1.5),
     # tile-edge sizes
     Workload("b_s2", 1, 2, 2, 2, 2, 128, seed=83, causal=True),
     Workload("b_s64", 1, 2, 1, 64, 64, 128, seed=84, causal=True),
@@ -239,11 +249,13 @@ def test_strided_inputs_match_contiguous():
     assert np.abs(lse.double().cpu().numpy() - lse_ref).max() <= 1e-3
 
 
-def test_guard_rows_are_untouched():
-    """O and LSE live inside larger buffers; the rows before and after must keep their pattern."""
+@pytest.mark.parametrize("hq,hkv,d", [(2, 2, 128), (4, 2, 128), (4, 1, 64), (2, 2, 256)])
+def test_guard_rows_are_untouched(hq, hkv, d):
+    """O and LSE live inside larger buffers; the rows before and after must keep their pattern (with an even GQA
+    group the output leaves through TMA tile stores of 32 rows, which must clip at row Sq = 200)."""
     import paper_2605_05023_b200 as pk
     dev = torch.device("cuda:0")
-    w = Workload("b_guard", 1, 2, 2, 200, 200, 128, seed=52, causal=True)
+    w = Workload("b_guard", 1, hq, hkv, 200, 200, d, seed=52, causal=True)
     q, k, v = make_qkv(w)
     n = w.B * w.Hq * w.Sq
     big_o = torch.full((n + 256, w.D), 7.0, device=dev, dtype=torch.bfloat16)
