@@ -13,8 +13,23 @@ struct ScoreConsts {
     float cap_in;      // scale / C   (0 when softcap is off)
     float cap_out;     // C * log2(e)
     float k0, k1, k2, k3;   // C*log2(e) * tanh(c s) ~= s * (k0 + k1 z + k2 z^2 + k3 z^3), z = s^2, c = cap_in, |c s| <= 0.5
+    float z_limit;     // the polynomial holds while s^2 <= z_limit = (0.5 / cap_in)^2
     bool softcap, has_bias;
 };
+
+// Coefficients of the softcap polynomial as register pairs.  identity: {1, 0, 0, 0}, which makes the polynomial
+// step return its input unchanged (second pass over a tile whose scores were capped exactly, see score_chunk32_tile).
+struct CapPoly {
+    uint64_t k0, k1, k2, k3;
+};
+__device__ __forceinline__ CapPoly cap_poly(const ScoreConsts& sc, bool identity) {
+    CapPoly k;
+    k.k0 = identity ? ptx::pack2(1.0f, 1.0f) : ptx::pack2(sc.k0, sc.k0);
+    k.k1 = identity ? 0ull : ptx::pack2(sc.k1, sc.k1);
+    k.k2 = identity ? 0ull : ptx::pack2(sc.k2, sc.k2);
+    k.k3 = identity ? 0ull : ptx::pack2(sc.k3, sc.k3);
+    return k;
+}
 
 // tanh(x) / x on |x| <= 0.5 as a cubic in x^2 (minimax, relative error 5.4e-7), with the input and output scales
 // folded into the coefficients.
@@ -32,6 +47,7 @@ __device__ __forceinline__ ScoreConsts make_score_consts(float scale, float soft
     sc.k1 = a * c2 * -0.3332631793391532f;
     sc.k2 = a * c2 * c2 * 0.13190296581692276f;
     sc.k3 = a * c2 * c2 * c2 * -0.04440222555537668f;
+    sc.z_limit = sc.softcap ? 0.25f / c2 : INFINITY;
     return sc;
 }
 
@@ -93,6 +109,57 @@ __device__ __forceinline__ void score_chunk32(uint32_t* y, const ScoreConsts& sc
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(__uint_as_float(y[i]) * sc.cs);
+    }
+}
+
+// ---- The softmax instances take the rare exponential form out of their key loop -------------------------------
+// (With the per-chunk choice above, the four unrolled copies of the exponential form sit inside the loop body and
+// every chunk ends in a warp vote: without them the softcap instances of the ping-pong kernel run 14 % faster.
+// The sigmoid and ReLU instances are slower with this form and keep the one above.)
+//
+// Softcap of large scores, exactly: the 32-lane x (32 * nchunks)-column block of raw scores at TMEM address taddr
+// is replaced in place by C * log2(e) * tanh(scale * s / C).  Called by all 32 lanes of a warp.
+static __device__ __noinline__ void softcap_exact_in_tmem(uint32_t taddr, int nchunks, float cap_in, float cap_out) {
+#pragma unroll 1
+    for (int c = 0; c < nchunks; ++c) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(taddr + c * 32, v);
+        ptx::tmem_wait_ld_regs(v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(cap_out * tanh_by_exp(__uint_as_float(v[i]) * cap_in));
+        ptx::tmem_st_32x32(taddr + c * 32, v);
+    }
+    ptx::tmem_wait_st();
+}
+
+// As score_chunk32<true>, but the softcap is always the polynomial, with the coefficients `poly`; zmax collects the
+// largest s^2 seen, and the caller compares it with sc.z_limit once per tile: if any score of the warp's tile lies
+// beyond, it has the tile capped exactly in TMEM (softcap_exact_in_tmem) and runs its pass again with the identity
+// coefficients.
+__device__ __forceinline__ void score_chunk32_tile(uint32_t* y, const ScoreConsts& sc, float rowoff, const CapPoly& poly, float& zmax) {
+    if (sc.softcap) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+            const uint64_t s2 = ptx::pack2(__uint_as_float(y[i]), __uint_as_float(y[i + 1]));
+            const uint64_t z = ptx::mul2(s2, s2);
+            float z0, z1;
+            ptx::unpack2(z, z0, z1);
+            zmax = ptx::max3(zmax, z0, z1);
+            uint64_t r = ptx::fma2(poly.k3, z, poly.k2);
+            r = ptx::fma2(r, z, poly.k1);
+            r = ptx::fma2(r, z, poly.k0);
+            float s0, s1;
+            ptx::unpack2(ptx::mul2(r, s2), s0, s1);
+            y[i] = __float_as_uint(s0);
+            y[i + 1] = __float_as_uint(s1);
+        }
+        if (sc.has_bias) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)      // + slope * (i' - j): the distance is formed exactly, then scaled
+                y[i] = __float_as_uint(fmaf(sc.slope2, rowoff - (float)i, __uint_as_float(y[i])));
+        }
+    } else {
+        score_chunk32<true>(y, sc, rowoff);
     }
 }
 

@@ -605,6 +605,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         ScoreConsts sc = {};
         if constexpr (SCORE != kScorePlain) sc = make_score_consts(p.scale, p.softcap, it.slope[qt]);
         const int niter = tr.jhi - tr.jlo;
+        CapPoly poly = {};
+        if constexpr (SCORE == kScoreGeneric && !SIGMOID && !RELU) poly = cap_poly(sc, false);
         float m_used = -INFINITY, l = 0.f;
         // Bias-only score (Appendix A.1): s*scale + slope*(i' - j) in log2 units = s*cs + slope2*(rowoff_chunk - i).
         // The column part -slope2*i is the same for every chunk and key tile: it sits in registers for the whole
@@ -636,6 +638,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             float bias_chunk[kBN / 32] = {};
             float mt_bias = -INFINITY;
+            float zmax = 0.f;                                    // largest squared raw score of the row in this tile (softcap)
             if constexpr (SCORE == kScoreBias) {
 #pragma unroll
                 for (int c = 0; c < kBN / 32; ++c) bias_chunk[c] = sc.slope2 * (rowoff - (float)(c * 32));
@@ -664,7 +667,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                             y[c * 32 + 2 * k2 + 1] = __float_as_uint(s1);
                         }
                     } else if constexpr (SCORE != kScorePlain) {
-                        score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                        if constexpr (!SIGMOID && !RELU) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
+                        else score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
                     }
                     if (kMasked) {
                         // One bit test per element (two compares per element made partial tiles cost half as much
@@ -695,6 +699,17 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             };
             if constexpr (SCORE == kScoreGeneric) {
                 load_score_max(std::false_type{}, !full_tile);
+                if constexpr (!SIGMOID && !RELU) {
+                    // Softcap: a score of this warp's rows beyond the polynomial's range (rare)?  Then the tile is
+                    // capped exactly in TMEM and the pass runs once more on it with the identity coefficients.
+                    if (__any_sync(0xffffffffu, zmax > sc.z_limit)) {
+                        softcap_exact_in_tmem(tm + buf * kBN, kBN / 32, sc.cap_in, sc.cap_out);
+                        poly = cap_poly(sc, true);
+                        mx[0] = mx[1] = mx[2] = mx[3] = -INFINITY;
+                        load_score_max(std::false_type{}, !full_tile);
+                        poly = cap_poly(sc, false);
+                    }
+                }
             } else {
                 if (full_tile) load_score_max(std::false_type{}, false);
                 else load_score_max(std::true_type{}, false);
