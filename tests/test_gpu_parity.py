@@ -445,6 +445,54 @@ def test_paper_model_configurations_sampled_rows(base):
             assert err_l <= tol_l, f"{w.name}: max|dLSE| = {err_l:.3e}"
 
 
+# ------------------------------------------------------------------ softcap: a few scores beyond the polynomial's range
+# The softmax instances cap with a polynomial tanh that holds while |scale * s / C| <= 0.5 and check the range once
+# per key tile; a tile with a score beyond it is capped exactly and passed over again.  Here a handful of keys is
+# scaled up so that only the key tiles that hold them (and there only the warps whose rows score high on them) take
+# that path, next to tiles that stay on the polynomial, with and without a position bias, at every head dimension.
+@pytest.mark.parametrize("w", [
+    Workload("cap_mixed_d128", 1, 4, 2, 900, 900, 128, seed=140, causal=True, softcap=30.0),
+    Workload("cap_mixed_d128_alibi", 1, 2, 2, 900, 900, 128, seed=141, causal=True, softcap=30.0, slopes=(-0.25, -0.0625)),
+    Workload("cap_mixed_d64", 1, 2, 1, 700, 700, 64, seed=142, softcap=20.0, window_left=300, window_right=300),
+    Workload("cap_mixed_d256", 1, 2, 2, 640, 640, 256, seed=143, causal=True, softcap=100.0, std=1.5),
+    Workload("cap_mixed_d256_fixed_reference", 1, 1, 1, 640, 640, 256, seed=144, causal=True, softcap=40.0, std=1.5),
+], ids=lambda w: w.name)
+def test_softcap_with_a_few_scores_beyond_the_polynomial_range(w):
+    q, k, v = make_qkv(w)
+    k = k.clone()
+    k[:, :, 130:134, :] *= 12.0            # one key tile of every head ...
+    k[:, :, 517, :] *= 20.0                # ... and a single key further on
+    raw = torch.einsum("bhid,bhjd->bhij", q.float()[:, ::w.Hq // w.Hkv], k.float()) * (w.scale or w.D ** -0.5)
+    frac = float((raw.abs() > 0.5 * w.softcap).float().mean())
+    assert 0.0 < frac < 0.02, f"{w.name}: the case must mix both paths (fraction beyond the range {frac:.4f})"
+    o, lse = gpu_run(w, q, k, v)
+    o_ref, lse_ref = oracle_run(w, q, k, v)
+    tol_o, tol_l = TOL[w.dtype]
+    assert np.abs(o.double().cpu().numpy() - o_ref).max() <= tol_o
+    assert np.abs(lse.double().cpu().numpy() - lse_ref).max() <= tol_l
+
+
+# ------------------------------------------------------------------ long sequences
+# 65 536 tokens per head (512 key tiles per work item at the end of a causal mask; with two heads per work item, more
+# query blocks per head than the heaviest-first table of the packed-document order holds, so that order falls back to
+# the plain one), sampled rows.
+LONG_CASES = [
+    Workload("long_causal", 1, 2, 1, 65536, 65536, 128, seed=150, causal=True),
+    Workload("long_window_alibi", 1, 4, 2, 65536, 65536, 128, seed=151, causal=True, window_left=4095, window_right=0,
+             slopes=(-0.5, -0.125, -0.03125, -0.0078125)),
+    Workload("long_docs_d256", 1, 1, 1, 65536, 65536, 256, seed=152, causal=True, std=1.5,
+             cu_seqlens=(0, 5000, 5001, 30000, 30130, 65536)),
+    Workload("long_docs_d128", 1, 2, 1, 65536, 65536, 128, seed=153, causal=True,
+             cu_seqlens=(0, 5000, 5001, 30000, 30130, 65536)),
+    Workload("long_cross", 1, 2, 2, 300, 65536, 64, seed=154),
+]
+
+
+@pytest.mark.parametrize("w", LONG_CASES, ids=lambda w: w.name)
+def test_long_sequences_sampled_rows(w):
+    check(w, rows=sampled_rows(w, 24, 1, seed=sum(map(ord, w.name)), every_head=8))
+
+
 # ------------------------------------------------------------------ masked positions have no influence (on the GPU)
 # Large finite garbage (+-1e4) is written into K and V at a band of key positions; every query row that cannot see
 # any key of the band must come out bit-identical to the clean run (a partial tile multiplies P = 0 by whatever V
