@@ -132,12 +132,43 @@ static __device__ __noinline__ void softcap_exact_in_tmem(uint32_t taddr, int nc
     ptx::tmem_wait_st();
 }
 
-// As score_chunk32<true>, but the softcap is always the polynomial, with the coefficients `poly`; zmax collects the
-// largest s^2 seen, and the caller compares it with sc.z_limit once per tile: if any score of the warp's tile lies
-// beyond, it has the tile capped exactly in TMEM (softcap_exact_in_tmem) and runs its pass again with the identity
-// coefficients.
+// The pieces of the softcap score on one chunk.  Polynomial with the item's own coefficients; zmax as above.
+__device__ __forceinline__ void softcap_poly_chunk32(uint32_t* y, const ScoreConsts& sc, float& zmax) {
+    const uint64_t k0 = ptx::pack2(sc.k0, sc.k0), k1 = ptx::pack2(sc.k1, sc.k1), k2 = ptx::pack2(sc.k2, sc.k2),
+                   k3 = ptx::pack2(sc.k3, sc.k3);
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const uint64_t s2 = ptx::pack2(__uint_as_float(y[i]), __uint_as_float(y[i + 1]));
+        const uint64_t z = ptx::mul2(s2, s2);
+        float z0, z1;
+        ptx::unpack2(z, z0, z1);
+        zmax = ptx::max3(zmax, z0, z1);
+        uint64_t r = ptx::fma2(k3, z, k2);
+        r = ptx::fma2(r, z, k1);
+        r = ptx::fma2(r, z, k0);
+        float s0, s1;
+        ptx::unpack2(ptx::mul2(r, s2), s0, s1);
+        y[i] = __float_as_uint(s0);
+        y[i + 1] = __float_as_uint(s1);
+    }
+}
+// Exponential form, any magnitude (raw scores in).
+__device__ __forceinline__ void softcap_exact_chunk32(uint32_t* y, const ScoreConsts& sc) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(sc.cap_out * tanh_by_exp(__uint_as_float(y[i]) * sc.cap_in));
+}
+// + slope * (i' - j): the distance is formed exactly, then scaled.
+__device__ __forceinline__ void bias_add_chunk32(uint32_t* y, const ScoreConsts& sc, float rowoff) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = __float_as_uint(fmaf(sc.slope2, rowoff - (float)i, __uint_as_float(y[i])));
+}
+
+// Softcap (always on in the instances that call this) and bias of one chunk, the softcap as the polynomial with the
+// coefficients `poly`; zmax collects the largest s^2 seen, and the caller compares it with sc.z_limit once per tile:
+// if any score of the warp's tile lies beyond, it has the tile capped exactly in TMEM (softcap_exact_in_tmem) and
+// runs its pass again with the identity coefficients.
 __device__ __forceinline__ void score_chunk32_tile(uint32_t* y, const ScoreConsts& sc, float rowoff, const CapPoly& poly, float& zmax) {
-    if (sc.softcap) {
+    {
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
             const uint64_t s2 = ptx::pack2(__uint_as_float(y[i]), __uint_as_float(y[i + 1]));
@@ -153,13 +184,7 @@ __device__ __forceinline__ void score_chunk32_tile(uint32_t* y, const ScoreConst
             y[i] = __float_as_uint(s0);
             y[i + 1] = __float_as_uint(s1);
         }
-        if (sc.has_bias) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)      // + slope * (i' - j): the distance is formed exactly, then scaled
-                y[i] = __float_as_uint(fmaf(sc.slope2, rowoff - (float)i, __uint_as_float(y[i])));
-        }
-    } else {
-        score_chunk32<true>(y, sc, rowoff);
+        if (sc.has_bias) bias_add_chunk32(y, sc, rowoff);
     }
 }
 

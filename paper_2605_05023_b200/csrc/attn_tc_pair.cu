@@ -546,10 +546,31 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             ptx::tmem_ld_32x32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&y[32]));
             ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[0]));
             ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[32]));
+            // Score (Appendix A.1).  Softcap in the softmax instances: the polynomial tanh on all columns and one range
+            // check per tile; if a score of this warp's columns lies beyond the polynomial's range (rare), the raw
+            // scores are read again and capped through the exponential form.
+            // (These instances are launched with a softcap only.)
+            constexpr bool kTileCap = (SCORE == kScoreGeneric) && !SIGMOID && !RELU;
+            if constexpr (kTileCap) {
+                float zmax = 0.f;
+#pragma unroll
+                for (int c = 0; c < kWgCols / 32; ++c) softcap_poly_chunk32(&y[c * 32], sc, zmax);
+                if (__any_sync(0xffffffffu, zmax > sc.z_limit)) {
+                    ptx::tmem_ld_32x32(ts, *reinterpret_cast<uint32_t(*)[32]>(&y[0]));
+                    ptx::tmem_ld_32x32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&y[32]));
+                    ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[0]));
+                    ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[32]));
+#pragma unroll
+                    for (int c = 0; c < kWgCols / 32; ++c) softcap_exact_chunk32(&y[c * 32], sc);
+                }
+                if (sc.has_bias) {
+#pragma unroll
+                    for (int c = 0; c < kWgCols / 32; ++c) bias_add_chunk32(&y[c * 32], sc, rowoff - (float)(c * 32));
+                }
+            }
 #pragma unroll
             for (int c = 0; c < kWgCols / 32; ++c) {
-                // Score (Appendix A.1)
-                if constexpr (SCORE != kScorePlain) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                if constexpr (SCORE != kScorePlain && !kTileCap) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
                 if (!full_tile) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);   // (the bit-test form cost this kernel 2 %)
                 if (!SIGMOID && !RELU && !fixed_max) {
 #pragma unroll
