@@ -845,8 +845,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                     }
                 }
             } else {
-                // bf16 output, two heads x 128 rows per item (both tiles end together and their epilogues compete
-                // for the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
+                // bf16 output, two heads x 128 rows per item or 256 rows without a mask (both tiles end together and
+                // their epilogues compete for the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
                 // in shared memory (64-byte swizzle: the 16-byte piece k of row r sits at piece k ^ ((r >> 1) & 3),
                 // conflict free) and leave as one TMA tile store, which also clips rows beyond Sq.  A thread-owns-a-row
                 // store to global memory touches 32 lines per instruction; this way the stores cost the load/store
@@ -881,7 +881,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 // kernel
 // ------------------------------------------------------------------------------------------------
 // GLB: masks with global tokens (two key pieces per row).  TMA_OUT: bf16 output through shared memory and TMA tile
-// stores (work items of two heads x 128 rows).
+// stores (work items whose two query tiles end together: two heads x 128 rows, or 256 rows without a mask).
 template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
 __global__ void __launch_bounds__(Cfg<D, NQ>::kThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
