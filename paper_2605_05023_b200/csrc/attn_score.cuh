@@ -132,7 +132,8 @@ static __device__ __noinline__ void softcap_exact_in_tmem(uint32_t taddr, int nc
     ptx::tmem_wait_st();
 }
 
-// The pieces of the softcap score on one chunk.  Polynomial with the item's own coefficients; zmax as above.
+// The pieces of the softcap score on one chunk.  Polynomial with the item's own coefficients; zmax collects the
+// largest s^2 seen (the caller compares it with sc.z_limit once per tile and caps exactly where it is exceeded).
 __device__ __forceinline__ void softcap_poly_chunk32(uint32_t* y, const ScoreConsts& sc, float& zmax) {
     const uint64_t k0 = ptx::pack2(sc.k0, sc.k0), k1 = ptx::pack2(sc.k1, sc.k1), k2 = ptx::pack2(sc.k2, sc.k2),
                    k3 = ptx::pack2(sc.k3, sc.k3);
