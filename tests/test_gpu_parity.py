@@ -232,6 +232,34 @@ def test_constant_v_and_rerun_is_bit_identical():
     assert float((o1.float() - 0.375).abs().max()) <= 2e-3    # bf16 rounding of sum(p_bf16)/sum(p)
 
 
+def test_launches_on_two_streams_at_once_match_the_serial_results():
+    """Two different kernels (ping-pong, D = 128; CTA pairs, D = 256) launched alternately on two streams with no
+    synchronisation in between: grids of both are resident together and every CTA takes further work items of its
+    own grid from the hardware scheduler.  Each launch must report no error and leave the bits of the serial run."""
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    wa = Workload("b_streams_a", 2, 8, 4, 2048, 2048, 128, seed=160, causal=True)
+    wb = Workload("b_streams_b", 1, 4, 4, 1536, 1536, 256, seed=161, causal=True, softcap=50.0, std=1.5)
+    runs = []
+    for w in (wa, wb):
+        q, k, v = (t.to(dev) for t in make_qkv(w))
+        o_ref, l_ref = pk.attn_fwd(q, k, v, **pk.variant_kwargs(w, dev))
+        torch.cuda.synchronize()
+        runs.append((w, q, k, v, o_ref.clone(), l_ref.clone(), torch.cuda.Stream(device=dev)))
+    outs = []
+    for rep in range(12):
+        for w, q, k, v, o_ref, l_ref, st in runs:
+            status = torch.zeros(1, dtype=torch.int32, device=dev)
+            o = torch.full_like(o_ref, float("nan"))
+            st.wait_stream(torch.cuda.current_stream(dev))      # the fills above run on the current stream
+            o, lse = pk.attn_fwd(q, k, v, o=o, status_word=status, stream=st, **pk.variant_kwargs(w, dev))
+            outs.append((o, lse, status, o_ref, l_ref))
+    torch.cuda.synchronize()
+    for o, lse, status, o_ref, l_ref in outs:
+        assert int(status.item()) == 0
+        assert torch.equal(o, o_ref) and torch.equal(lse, l_ref)
+
+
 def test_strided_inputs_match_contiguous():
     """q, k, v given as [B, S, H, D] storage viewed as [B, H, S, D] (strides in the descriptor)."""
     import paper_2605_05023_b200 as pk
