@@ -5,6 +5,7 @@
 // [lo, hi].  hi is non-decreasing in the row index; lo is non-decreasing too, except
 // that it falls back to the window / sequence start at row test_query_start.
 #pragma once
+#include <algorithm>
 #include <cstdint>
 #include <cuda_runtime.h>
 
@@ -40,6 +41,7 @@ struct AttnParams {
     int test_query_start;       // rows i >= this ignore the document clause (Sq = none)
     int global_len;             // global tokens: positions < global_len pass the window / document clauses (0 = none)
     int head_pair;              // ping-pong kernel: a work item is two heads x 128 rows (1) or one head x 256 rows (0)
+    int defer_blocks;           // ping-pong kernel: query blocks per head whose work items end the work order (see decode_item)
 };
 
 struct RowInterval {
@@ -133,6 +135,36 @@ __device__ __forceinline__ TileBounds tile_bounds(const AttnParams& p, int q0, i
     }
     t.any = !(t.hi_max < 0 || t.lo_min > t.hi_max) || t.pre_max > 0;
     return t;
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+// How many of the first (lightest) query blocks of every head go to the end of the work order (decode_item of the
+// ping-pong and of the CTA-pair kernel).  Causal masks without documents or global tokens only: there a block's key
+// tiles grow with its index, and the count follows from the row intervals.  `rows`: query rows of a work item;
+// `key_tile`: keys per key tile; `workers`: CTAs (or CTA pairs) that run at once.  As many blocks as hold about
+// 0.6 x workers x (heaviest item) key tiles of work, at most a quarter of all work and half of the blocks; none when
+// the items do not differ by a factor of two (equal items need no filler).
+inline int deferred_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long items_per_block, int workers) {
+    if (!(p.mask_flags & kMaskCausal) || (p.mask_flags & (kMaskDocument | kMaskGlobal)) || nqb < 4) return 0;
+    auto tiles = [&](int qb) -> long long {           // key tiles of the block's item (union over its rows)
+        const long long first = (long long)qb * rows + p.Sk - p.Sq;
+        const long long last = std::min<long long>((long long)(qb + 1) * rows, p.Sq) - 1 + p.Sk - p.Sq;
+        long long hi = std::max<long long>(last, (long long)p.prefix_len - 1);
+        hi = std::min<long long>(hi, p.Sk - 1);
+        long long lo = 0;
+        if ((p.mask_flags & kMaskWindow) && p.window_left >= 0) lo = std::max<long long>(0, first - p.window_left);
+        if (p.prefix_len > 0 && first < p.prefix_len) lo = 0;
+        if (hi < 0 || lo > hi) return 0;
+        return hi / key_tile - lo / key_tile + 1;
+    };
+    long long total = 0, w_max = 0, w_min = 1ll << 40;
+    for (int qb = 0; qb < nqb; ++qb) { const long long w = tiles(qb); total += w; w_max = std::max(w_max, w); w_min = std::min(w_min, w); }
+    if (w_max < 2 * std::max<long long>(w_min, 1)) return 0;
+    const long long target = std::min(total * items_per_block / 4, (long long)workers * w_max * 6 / 10);
+    long long cum = 0;
+    int d = 0;
+    while (d < nqb / 2 && cum < target) { cum += tiles(d) * items_per_block; ++d; }
+    return d;
 }
 
 }  // namespace b200attn

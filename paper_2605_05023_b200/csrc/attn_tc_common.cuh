@@ -3,6 +3,7 @@
 // partial tile, the exponential step of the online softmax, and the host-side TMA tensor maps.  (Bounded waits,
 // the work-item fetch and the warp-level arrivals are in sm100_sync.cuh.)
 #pragma once
+#include <algorithm>
 #include <atomic>
 
 #include <cuda.h>
@@ -89,6 +90,19 @@ inline bool set_smem_attr_once(SmemAttrFlags& done, Kernel kernel, int bytes) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
     if (tracked) done[dev].store(true, std::memory_order_release);
     return true;
+}
+
+// SMs of the current device (cached per device; 148 on a B200), for the kernels' work-order heuristics.
+inline int device_sm_count() {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    const bool tracked = dev >= 0 && dev < 64;
+    if (tracked) { const int c = cached[dev].load(std::memory_order_acquire); if (c > 0) return c; }
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    if (tracked) cached[dev].store(n, std::memory_order_release);
+    return n;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -117,17 +117,28 @@ __device__ __forceinline__ TileRange pair_range(const AttnParams& p, int q0) {
 
 // Work item of a pair index.  Heads are taken in sections whose K/V fit in L2; inside a section the query
 // block index is the slow coordinate and runs from the last block (most keys under a causal mask) to the
-// first, so the hardware hands out the heaviest items first.
+// first, so the hardware hands out the heaviest items first.  The p.defer_blocks first (lightest) blocks of every
+// head come after all sections, again heaviest first: they fill in the end of the grid, where the last section's
+// long items would otherwise leave the pairs' finish times up to one long item apart.
 __device__ __forceinline__ Item decode_item(const AttnParams& p, int pair) {
     const int nqb = (p.Sq + 2 * kBM - 1) / (2 * kBM);
     const int bh_total = p.B * p.Hq;
-    const int per_sec = p.sec_heads * nqb;
-    const int sec = pair / per_sec;
-    const int r = pair - sec * per_sec;
-    const int sec_start = sec * p.sec_heads;
-    const int sh = min(p.sec_heads, bh_total - sec_start);
-    const int qb = nqb - 1 - r / sh;
-    const int bh = sec_start + r % sh;
+    const int nh = nqb - p.defer_blocks;                 // blocks per head that are taken section by section
+    int rank, bh;
+    if (pair < bh_total * nh) {
+        const int per_sec = p.sec_heads * nh;
+        const int sec = pair / per_sec;
+        const int r = pair - sec * per_sec;
+        const int sec_start = sec * p.sec_heads;
+        const int sh = min(p.sec_heads, bh_total - sec_start);
+        rank = r / sh;
+        bh = sec_start + r % sh;
+    } else {                                             // the deferred blocks: one last section of all heads
+        const int r = pair - bh_total * nh;
+        rank = nh + r / bh_total;
+        bh = r % bh_total;
+    }
+    const int qb = nqb - 1 - rank;
     Item it;
     it.b = bh / p.Hq;
     it.h = bh - it.b * p.Hq;
@@ -865,6 +876,7 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     const long long nqb = (p.Sq + 2 * kBM - 1) / (2 * kBM);
     const long long grid = 2 * nqb * bh;
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
+    p.defer_blocks = deferred_blocks(p, 2 * kBM, kBN, (int)nqb, bh, device_sm_count() / 2);
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
