@@ -142,8 +142,8 @@ __device__ __forceinline__ TileBounds tile_bounds(const AttnParams& p, int q0, i
 // ping-pong and of the CTA-pair kernel).  Causal masks without documents or global tokens only: there a block's key
 // tiles grow with its index, and the count follows from the row intervals.  `rows`: query rows of a work item;
 // `key_tile`: keys per key tile; `workers`: CTAs (or CTA pairs) that run at once.  As many blocks as hold about
-// 0.6 x workers x (heaviest item) key tiles of work, at most a quarter of all work and half of the blocks; none when
-// the items do not differ by a factor of two (equal items need no filler).
+// 0.6 x workers x (heaviest item) key tiles of work, at most half of the blocks; none when that is more than a quarter
+// of all work (a small grid) or when the items do not differ by a factor of two (equal items need no filler).
 inline int deferred_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long items_per_block, int workers) {
     if (!(p.mask_flags & kMaskCausal) || (p.mask_flags & (kMaskDocument | kMaskGlobal)) || nqb < 4) return 0;
     auto tiles = [&](int qb) -> long long {           // key tiles of the block's item (union over its rows)
@@ -160,7 +160,8 @@ inline int deferred_blocks(const AttnParams& p, int rows, int key_tile, int nqb,
     long long total = 0, w_max = 0, w_min = 1ll << 40;
     for (int qb = 0; qb < nqb; ++qb) { const long long w = tiles(qb); total += w; w_max = std::max(w_max, w); w_min = std::min(w_min, w); }
     if (w_max < 2 * std::max<long long>(w_min, 1)) return 0;
-    const long long target = std::min(total * items_per_block / 4, (long long)workers * w_max * 6 / 10);
+    const long long target = (long long)workers * w_max * 6 / 10;
+    if (target > total * items_per_block / 4) return 0;      // a small grid: the "filler" would be most of the work
     long long cum = 0;
     int d = 0;
     while (d < nqb / 2 && cum < target) { cum += tiles(d) * items_per_block; ++d; }
