@@ -41,7 +41,7 @@ struct AttnParams {
     int test_query_start;       // rows i >= this ignore the document clause (Sq = none)
     int global_len;             // global tokens: positions < global_len pass the window / document clauses (0 = none)
     int head_pair;              // ping-pong kernel: a work item is two heads x 128 rows (1) or one head x 256 rows (0)
-    int defer_blocks;           // ping-pong kernel: query blocks per head whose work items end the work order (see decode_item)
+    int defer_blocks;           // tensor-core kernels: query blocks per head whose work items end the work order (see work_order)
 };
 
 struct RowInterval {
@@ -135,6 +135,28 @@ __device__ __forceinline__ TileBounds tile_bounds(const AttnParams& p, int q0, i
     }
     t.any = !(t.hi_max < 0 || t.lo_min > t.hi_max) || t.pre_max > 0;
     return t;
+}
+
+// Work order of the tensor-core kernels: the (batch, head) unit and the query block of linear work index `lin`.
+// Units are taken in sections of `sec_units` whose K/V fit in L2; inside a section the query block is the slow
+// coordinate and runs from the heaviest block of a unit (rank 0) to the lightest, so the hardware hands out the
+// heaviest items first.  The `defer` lightest blocks of every unit come after all sections, again heaviest first
+// (see deferred_blocks).  rank: position of the block among its unit's `nqb` blocks, heaviest first.
+__device__ __forceinline__ void work_order(int lin, int units_total, int sec_units, int nqb, int defer, int& rank, int& unit) {
+    const int nh = nqb - defer;                          // blocks per unit that are taken section by section
+    if (lin < units_total * nh) {
+        const int per_sec = sec_units * nh;
+        const int sec = lin / per_sec;
+        const int r = lin - sec * per_sec;
+        const int sec_start = sec * sec_units;
+        const int sh = min(sec_units, units_total - sec_start);
+        rank = r / sh;
+        unit = sec_start + r % sh;
+    } else {                                             // the deferred blocks: one last section of all units
+        const int r = lin - units_total * nh;
+        rank = nh + r / units_total;
+        unit = r % units_total;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ host side

@@ -115,29 +115,13 @@ __device__ __forceinline__ TileRange pair_range(const AttnParams& p, int q0) {
     return TileRange{t.lo_min / kBN, t.hi_max / kBN + 1};
 }
 
-// Work item of a pair index.  Heads are taken in sections whose K/V fit in L2; inside a section the query
-// block index is the slow coordinate and runs from the last block (most keys under a causal mask) to the
-// first, so the hardware hands out the heaviest items first.  The p.defer_blocks first (lightest) blocks of every
-// head come after all sections, again heaviest first: they fill in the end of the grid, where the last section's
-// long items would otherwise leave the pairs' finish times up to one long item apart.
+// Work item of a pair index (work_order in attn_params.cuh: sections of heads whose K/V fit in L2, last query block
+// first, the first blocks of every head at the very end).
 __device__ __forceinline__ Item decode_item(const AttnParams& p, int pair) {
     const int nqb = (p.Sq + 2 * kBM - 1) / (2 * kBM);
     const int bh_total = p.B * p.Hq;
-    const int nh = nqb - p.defer_blocks;                 // blocks per head that are taken section by section
     int rank, bh;
-    if (pair < bh_total * nh) {
-        const int per_sec = p.sec_heads * nh;
-        const int sec = pair / per_sec;
-        const int r = pair - sec * per_sec;
-        const int sec_start = sec * p.sec_heads;
-        const int sh = min(p.sec_heads, bh_total - sec_start);
-        rank = r / sh;
-        bh = sec_start + r % sh;
-    } else {                                             // the deferred blocks: one last section of all heads
-        const int r = pair - bh_total * nh;
-        rank = nh + r / bh_total;
-        bh = r % bh_total;
-    }
+    work_order(pair, bh_total, p.sec_heads, nqb, p.defer_blocks, rank, bh);
     const int qb = nqb - 1 - rank;
     Item it;
     it.b = bh / p.Hq;

@@ -153,15 +153,10 @@ __device__ __forceinline__ TileRange tile_range(const AttnParams& p, int q0, int
     return TileRange{t.lo_min / kBN, t.hi_max / kBN + 1};
 }
 
-// Work item of a linear index.  Heads are taken in sections whose K/V fit in L2; inside a section the
-// query block index is the slow coordinate and runs from the last block (most keys under a causal mask)
-// to the first, so the hardware hands out the heaviest items first.
-// `order`, when not null, lists the query blocks of a head heaviest first (packed documents, see build_block_order);
-// otherwise the blocks are taken from the last to the first.
-// The p.defer_blocks lightest blocks of every head (the first ones; set by the launcher for causal masks) come after
-// all sections, again heaviest first: without them the grid would end with the last section's share of long items, at
-// most a few per SM, and the SMs' finish times would differ by up to one long item (c2 causal: 7 % of the SM cycles
-// idle at the end); the light items fill that in, and they read only the first keys of their head again.
+// Work item of a linear index (work_order in attn_params.cuh: sections of heads whose K/V fit in L2, heaviest query
+// block first, the lightest blocks of every head at the very end).  `order`, when not null, lists the query blocks of
+// a head heaviest first (packed documents, see build_block_order); otherwise the blocks are taken from the last to
+// the first (most keys under a causal mask).
 template <int NQ>
 __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const uint16_t* order) {
     // The two query tiles of an item share every K / V tile.  With an even GQA group they are the same 128 rows
@@ -174,21 +169,8 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     const int units = pair ? 2 : 1;                      // query heads per item
     const int bh_total = p.B * p.Hq / units;
     const int sec_units = p.sec_heads / units;
-    const int nh = nqb - p.defer_blocks;                 // blocks per head that are taken section by section
     int rank, bh;                                        // rank of the block among its head's blocks, heaviest first
-    if (lin < bh_total * nh) {
-        const int per_sec = sec_units * nh;
-        const int sec = lin / per_sec;
-        const int r = lin - sec * per_sec;
-        const int sec_start = sec * sec_units;
-        const int sh = min(sec_units, bh_total - sec_start);
-        rank = r / sh;
-        bh = sec_start + r % sh;
-    } else {                                             // the deferred blocks: one last section of all heads
-        const int r = lin - bh_total * nh;
-        rank = nh + r / bh_total;
-        bh = r % bh_total;
-    }
+    work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh);
     const int qb = order ? (int)order[rank] : nqb - 1 - rank;
     const int hq_units = p.Hq / units;
     ItemG it;

@@ -113,19 +113,14 @@ __device__ __forceinline__ TileRange tile_range(const AttnParams& p, int q0) {
     return TileRange{jlo, jhi, pend};
 }
 
-// Work item of a linear index.  Heads are taken in sections whose K/V fit in L2; inside a section the
-// query tile index is the slow coordinate and runs from the last tile (most keys under a causal mask)
-// to the first, so the hardware hands out the heaviest items first.
+// Work item of a linear index (work_order in attn_params.cuh: sections of heads whose K/V fit in L2, last query tile
+// first).
 __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
     const int nqb = (p.Sq + kBM - 1) / kBM;
     const int bh_total = p.B * p.Hq;
-    const int per_sec = p.sec_heads * nqb;
-    const int sec = lin / per_sec;
-    const int r = lin - sec * per_sec;
-    const int sec_start = sec * p.sec_heads;
-    const int sh = min(p.sec_heads, bh_total - sec_start);
-    const int qb = nqb - 1 - r / sh;
-    const int bh = sec_start + r % sh;
+    int rank, bh;
+    work_order(lin, bh_total, p.sec_heads, nqb, 0, rank, bh);      // (this kernel defers no blocks)
+    const int qb = nqb - 1 - rank;
     Item it;
     it.b = bh / p.Hq;
     it.h = bh - it.b * p.Hq;
