@@ -826,18 +826,25 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                                              __uint_as_float(orr[4 * i + 2]) * inv, __uint_as_float(orr[4 * i + 3]) * inv);
                 }
             } else if constexpr (!TMA_OUT) {
-                // bf16 output, 256 consecutive rows per item: the first tile's epilogue runs under the second tile's
-                // last key step and the threads go on at once, so plain 16-byte stores by the row's owner are best.
+                // bf16 output, 256 consecutive rows per item under a mask: the first tile's epilogue runs under the second
+                // tile's last key step and the threads go on at once, so plain stores by the row's owner are best:
+                // 32 bytes at a time (a whole sector per thread and instruction; with 16-byte stores the exposed epilogue
+                // of the second tile took 3.7 k cycles, nearly all of them in the load/store unit).
                 if (store_row) {
-                    uint4* dst = reinterpret_cast<uint4*>(obase + c * 64);
+                    char* dst = obase + c * 64;
+                    const bool aligned32 = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;     // (always, for dense rows)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 w;
-                        w.x = ptx::pack_bf16x2(__uint_as_float(orr[8 * i]) * inv, __uint_as_float(orr[8 * i + 1]) * inv);
-                        w.y = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 2]) * inv, __uint_as_float(orr[8 * i + 3]) * inv);
-                        w.z = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 4]) * inv, __uint_as_float(orr[8 * i + 5]) * inv);
-                        w.w = ptx::pack_bf16x2(__uint_as_float(orr[8 * i + 6]) * inv, __uint_as_float(orr[8 * i + 7]) * inv);
-                        dst[i] = w;
+                    for (int i = 0; i < 2; ++i) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int k2 = 0; k2 < 8; ++k2)
+                            w[k2] = ptx::pack_bf16x2(__uint_as_float(orr[16 * i + 2 * k2]) * inv, __uint_as_float(orr[16 * i + 2 * k2 + 1]) * inv);
+                        if (aligned32) {
+                            ptx::st_global_v8(dst + i * 32, w);
+                        } else {
+                            reinterpret_cast<uint4*>(dst + i * 32)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                            reinterpret_cast<uint4*>(dst + i * 32)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        }
                     }
                 }
             } else {

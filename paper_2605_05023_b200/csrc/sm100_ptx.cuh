@@ -60,6 +60,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const CUtensorMap
         : "memory");
 }
 
+// 32-byte store to global memory (sm_100: 256-bit vector stores); p must be 32-byte aligned.  A thread that writes a
+// row piece by piece fills a whole 32-byte sector per instruction this way, half as many trips through the load/store
+// unit as with 16-byte stores.
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+
 // TMA tile store (shared memory -> global), completion tracked by the issuing thread's bulk async-group.
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src_smem, int c0, int c1, int c2, int c3) {
     asm volatile(
