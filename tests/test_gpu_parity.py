@@ -260,6 +260,33 @@ def test_launches_on_two_streams_at_once_match_the_serial_results():
         assert torch.equal(o, o_ref) and torch.equal(lse, l_ref)
 
 
+@pytest.mark.parametrize("w", [
+    Workload("b_o_offset16_d128", 1, 3, 3, 300, 300, 128, seed=170, causal=True),
+    Workload("b_o_offset16_d256", 1, 2, 2, 300, 300, 256, seed=171, causal=True, std=1.5),
+    Workload("b_o_offset16_d256_fp32", 1, 1, 1, 300, 300, 256, seed=172, causal=True, normalizer="sigmoid", o_dtype="fp32",
+             sigmoid_bias=-math.log(300.0), std=1.5),
+], ids=lambda w: w.name)
+def test_output_that_is_only_16_byte_aligned(w):
+    """The rows that threads store themselves go out in 32-byte pieces when the output is 32-byte aligned; an output
+    tensor that starts 16 bytes into its storage takes the 16-byte form.  Guard elements around it stay untouched."""
+    import paper_2605_05023_b200 as pk
+    dev = torch.device("cuda:0")
+    q, k, v = make_qkv(w)
+    odt = torch.float32 if w.o_dtype == "fp32" else torch.bfloat16
+    n = w.B * w.Hq * w.Sq * w.D
+    off = 16 // torch.empty((), dtype=odt).element_size()
+    buf = torch.full((n + 2 * off,), 7.0, device=dev, dtype=odt)
+    o = buf[off:off + n].view(w.B, w.Hq, w.Sq, w.D)
+    assert o.data_ptr() % 32 == 16
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    o, lse = pk.attn_fwd(q.to(dev), k.to(dev), v.to(dev), o=o, status_word=status, **pk.variant_kwargs(w, dev))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    o_ref, lse_ref = oracle_run(w, q, k, v)
+    assert np.abs(o.double().cpu().numpy() - o_ref).max() <= TOL["bf16"][0]
+    assert bool((buf[:off] == 7.0).all()) and bool((buf[off + n:] == 7.0).all())
+
+
 def test_strided_inputs_match_contiguous():
     """q, k, v given as [B, S, H, D] storage viewed as [B, H, S, D] (strides in the descriptor)."""
     import paper_2605_05023_b200 as pk
