@@ -13,11 +13,10 @@ int launch_attn_fwd_bf16_pingpong_tmaout(const AttnParams& p, cudaStream_t strea
 
 namespace {
 // Masks with global tokens get their own instances, so that the others carry none of the two-piece walk; work items
-// whose two query tiles end together (two heads x 128 rows with an even GQA group; 256 rows without any mask) with bf16
-// output get the instances whose epilogue goes through TMA stores.
+// of two heads x 128 rows (even GQA group) with bf16 output get the instances whose epilogue goes through TMA stores.
 int launch_pingpong(const AttnParams& p, cudaStream_t stream) {
     if (p.mask_flags & kMaskGlobal) return launch_attn_fwd_bf16_pingpong_global(p, stream);
-    if ((p.group % 2 == 0 || p.mask_flags == 0) && !p.o_fp32) return launch_attn_fwd_bf16_pingpong_tmaout(p, stream);
+    if (p.group % 2 == 0 && !p.o_fp32) return launch_attn_fwd_bf16_pingpong_tmaout(p, stream);
     switch (p.D) {
         case 64: return launch_for_mask<64, 2, false, false>(p, stream);
         case 128: return launch_for_mask<128, 2, false, false>(p, stream);

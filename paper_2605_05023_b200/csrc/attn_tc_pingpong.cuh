@@ -826,8 +826,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                                              __uint_as_float(orr[4 * i + 2]) * inv, __uint_as_float(orr[4 * i + 3]) * inv);
                 }
             } else if constexpr (!TMA_OUT) {
-                // bf16 output, 256 consecutive rows per item under a mask: the first tile's epilogue runs under the second
-                // tile's last key step and the threads go on at once, so plain stores by the row's owner are best:
+                // bf16 output, 256 consecutive rows per item: under a causal mask the first tile's epilogue runs under the
+                // second tile's last key step, and the threads go on at once, so plain stores by the row's owner are best:
                 // 32 bytes at a time (a whole sector per thread and instruction; with 16-byte stores the exposed epilogue
                 // of the second tile took 3.7 k cycles, nearly all of them in the load/store unit).
                 if (store_row) {
@@ -848,8 +848,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                     }
                 }
             } else {
-                // bf16 output, two heads x 128 rows per item or 256 rows without a mask (both tiles end together and
-                // their epilogues compete for the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
+                // bf16 output, two heads x 128 rows per item (both tiles end together and their epilogues compete for
+                // the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
                 // in shared memory (64-byte swizzle: the 16-byte piece k of row r sits at piece k ^ ((r >> 1) & 3),
                 // conflict free) and leave as one TMA tile store, which also clips rows beyond Sq.  A thread-owns-a-row
                 // store to global memory touches 32 lines per instruction; this way the stores cost the load/store
@@ -884,7 +884,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 // kernel
 // ------------------------------------------------------------------------------------------------
 // GLB: masks with global tokens (two key pieces per row).  TMA_OUT: bf16 output through shared memory and TMA tile
-// stores (work items whose two query tiles end together: two heads x 128 rows, or 256 rows without a mask).
+// stores (work items of two heads x 128 rows).
 template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
 __global__ void __launch_bounds__(Cfg<D, NQ>::kThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
