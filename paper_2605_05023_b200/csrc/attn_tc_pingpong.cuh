@@ -601,8 +601,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         ScoreConsts sc = {};
         if constexpr (SCORE != kScorePlain) sc = make_score_consts(p.scale, p.softcap, it.slope[qt]);
         const int niter = tr.jhi - tr.jlo;
-        CapPoly poly = {};
-        if constexpr (SCORE == kScoreGeneric && !SIGMOID && !RELU) poly = cap_poly(sc, false);
+        CapPoly poly = {};                                   // softcap: coefficients of a tile's second pass
         float m_used = -INFINITY, l = 0.f;
         // Bias-only score (Appendix A.1): s*scale + slope*(i' - j) in log2 units = s*cs + slope2*(rowoff_chunk - i).
         // The column part -slope2*i is the same for every chunk and key tile: it sits in registers for the whole
@@ -642,8 +641,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             // Loading, score modifier, mask and row maximum, compiled twice: the copy for full tiles is straight-line
             // code without the mask blocks (for the softcap instance, whose score code is long, there is one copy
             // with a run-time test instead).
-            auto load_score_max = [&](auto masked_tag, bool masked_rt) {
+            auto load_score_max = [&](auto masked_tag, bool masked_rt, auto redo_tag) {
                 constexpr bool kTag = decltype(masked_tag)::value;
+                constexpr bool kRedo = decltype(redo_tag)::value;     // softcap: second pass over a tile (see below)
+                (void)kRedo;
                 const bool kMasked = kTag || masked_rt;
                 ptx::tmem_ld_32x32(tm + buf * kBN, *reinterpret_cast<uint32_t(*)[32]>(&y[0]));
                 ptx::tmem_wait_ld_regs(*reinterpret_cast<uint32_t(*)[32]>(&y[0]));
@@ -663,8 +664,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                             y[c * 32 + 2 * k2 + 1] = __float_as_uint(s1);
                         }
                     } else if constexpr (SCORE != kScorePlain) {
-                        if constexpr (!SIGMOID && !RELU) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
-                        else score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                        if constexpr (SIGMOID || RELU) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                        else if constexpr (kRedo) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
+                        else score_chunk32_quad(&y[c * 32], sc, rowoff - (float)(c * 32), zmax);
                     }
                     if (kMasked) {
                         // One bit test per element (two compares per element made partial tiles cost half as much
@@ -694,21 +696,22 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 }
             };
             if constexpr (SCORE == kScoreGeneric) {
-                load_score_max(std::false_type{}, !full_tile);
+                load_score_max(std::false_type{}, !full_tile, std::false_type{});
                 if constexpr (!SIGMOID && !RELU) {
-                    // Softcap: a score of this warp's rows beyond the polynomial's range (rare)?  Then the tile is
-                    // capped exactly in TMEM and the pass runs once more on it with the identity coefficients.
-                    if (__any_sync(0xffffffffu, zmax > sc.z_limit)) {
-                        softcap_exact_in_tmem(tm + buf * kBN, kBN / 32, sc.cap_in, sc.cap_out);
-                        poly = cap_poly(sc, true);
+                    // Softcap: the first pass caps with the quadratic (scores up to 0.35 of the cap).  A score of this
+                    // warp's rows beyond that (rare)?  Then the pass runs once more: with the cubic (up to half the
+                    // cap), or, beyond that too, on the tile capped exactly in TMEM with the identity coefficients.
+                    if (__any_sync(0xffffffffu, zmax > sc.zq_limit)) {
+                        const bool exact = __any_sync(0xffffffffu, zmax > sc.z_limit);
+                        if (exact) softcap_exact_in_tmem(tm + buf * kBN, kBN / 32, sc.cap_in, sc.cap_out);
+                        poly = cap_poly(sc, exact);
                         mx[0] = mx[1] = mx[2] = mx[3] = -INFINITY;
-                        load_score_max(std::false_type{}, !full_tile);
-                        poly = cap_poly(sc, false);
+                        load_score_max(std::false_type{}, !full_tile, std::true_type{});
                     }
                 }
             } else {
-                if (full_tile) load_score_max(std::false_type{}, false);
-                else load_score_max(std::true_type{}, false);
+                if (full_tile) load_score_max(std::false_type{}, false, std::false_type{});
+                else load_score_max(std::true_type{}, false, std::false_type{});
             }
             if constexpr (SIGMOID) {
                 // Appendix A.3: p = sigmoid(s + b); a masked score (-inf) gives exactly 0.  An unnormalised row can
