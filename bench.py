@@ -52,7 +52,7 @@ STEP_SETS = {
 # over its launches; None where no capture exists.
 NCU_TRAFFIC_BYTES_PER_VARIANT = {
     "c2_noncausal": 318.6e6, "c2_causal": 339.5e6, "c3_gqa_window_alibi": 308.7e6,
-    "c4a_softcap": 348.4e6, "c4b_sigmoid": 409.1e6, "c5_packed_doc_causal": 1152.1e6,
+    "c4a_softcap": 346.2e6, "c4b_sigmoid": 409.1e6, "c5_packed_doc_causal": 1152.1e6,
 }
 
 
