@@ -593,6 +593,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 // rides in the constants; the epilogue takes it out again together with out_scale).
                 const uint64_t nb2 = ptx::pack2(-sig_bias2 - 10.0f, -sig_bias2 - 10.0f), neg1 = ptx::pack2(-1.0f, -1.0f);
                 constexpr float kTwoToMinus10 = 0.0009765625f;
+                // Two special-function operations per score (ex2, rcp) make that unit the busiest at D = 128, where a key
+                // step has half the tensor work of D = 256: there every other pair of scores takes its reciprocal on
+                // the FMA pipe instead (sweep sigmoid rows +7 to 11 % at S <= 4k; at D = 256 the same costs c4b 2 %).
+                constexpr int kNewtonEvery = (D == 128) ? 2 : 0;
 #pragma unroll
                 for (int cc = 0; cc < kWgCols / 32; ++cc) {
                     uint32_t pk[16];
@@ -601,8 +605,24 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         const uint64_t yy = ptx::pack2(__uint_as_float(y[cc * 32 + 2 * i]), __uint_as_float(y[cc * 32 + 2 * i + 1]));
                         float z0, z1;
                         ptx::unpack2(ptx::fma2(yy, neg1, nb2), z0, z1);                  // -(s + b) in log2 units, - 10
-                        const float p0 = ptx::rcp_approx(kTwoToMinus10 + ptx::ex2_approx(z0));
-                        const float p1 = ptx::rcp_approx(kTwoToMinus10 + ptx::ex2_approx(z1));
+                        const float t0 = kTwoToMinus10 + ptx::ex2_approx(z0), t1 = kTwoToMinus10 + ptx::ex2_approx(z1);
+                        float p0, p1;
+                        if (kNewtonEvery > 0 && (i % kNewtonEvery) == 0) {
+                            // Reciprocal on the FMA pipe: bit-trick seed (12 % off at worst) and two Newton steps,
+                            // relative error 2.4e-4, half of what the fp16 rounding of P adds.
+                            // (A masked score arrives here as t = +inf: bounded, so that the steps stay finite; the
+                            // result, below 1e-30, still rounds to an fp16 zero.)
+                            const float u0 = fminf(t0, 1e30f), u1 = fminf(t1, 1e30f);
+                            const uint64_t nt2 = ptx::pack2(-u0, -u1), two2 = ptx::pack2(2.0f, 2.0f);
+                            uint64_t r = ptx::pack2(__int_as_float(0x7EF311C7 - __float_as_int(u0)),
+                                                    __int_as_float(0x7EF311C7 - __float_as_int(u1)));
+                            r = ptx::mul2(r, ptx::fma2(nt2, r, two2));
+                            r = ptx::mul2(r, ptx::fma2(nt2, r, two2));
+                            ptx::unpack2(r, p0, p1);
+                        } else {
+                            p0 = ptx::rcp_approx(t0);
+                            p1 = ptx::rcp_approx(t1);
+                        }
                         pk[i] = ptx::pack_f16x2(p0, p1);
                     }
                     ptx::tmem_st_32x16(ts + cc * 16, pk);
