@@ -573,7 +573,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             }
 #pragma unroll
             for (int c = 0; c < kWgCols / 32; ++c) {
-                if constexpr (SCORE != kScorePlain && !kTileCap) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                if constexpr (SCORE != kScorePlain && !kTileCap) {
+                    // (Sigmoid without softcap or bias: the scale rides in the sigmoid's own first FMA, below.)
+                    if (!(SIGMOID && !sc.softcap && !sc.has_bias)) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                }
                 if (!full_tile) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);   // (the bit-test form cost this kernel 2 %)
                 if (!SIGMOID && !RELU && !fixed_max) {
 #pragma unroll
@@ -591,7 +594,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 // be carried by a few large weights, so the 8 significant bits of a bf16 P would show in O: P is
                 // written as fp16, scaled by 2^10 (2^10 * sigmoid(x) = 1 / (2^-10 + 2^(-x log2 e - 10)): the scale
                 // rides in the constants; the epilogue takes it out again together with out_scale).
-                const uint64_t nb2 = ptx::pack2(-sig_bias2 - 10.0f, -sig_bias2 - 10.0f), neg1 = ptx::pack2(-1.0f, -1.0f);
+                const float neg_mul = (!sc.softcap && !sc.has_bias) ? -sc.cs : -1.0f;      // raw scores in, or scores in log2 units
+                const uint64_t nb2 = ptx::pack2(-sig_bias2 - 10.0f, -sig_bias2 - 10.0f), neg1 = ptx::pack2(neg_mul, neg_mul);
                 constexpr float kTwoToMinus10 = 0.0009765625f;
                 // Two special-function operations per score (ex2, rcp) make that unit the busiest at D = 128, where a key
                 // step has half the tensor work of D = 256: there every other pair of scores takes its reciprocal on
