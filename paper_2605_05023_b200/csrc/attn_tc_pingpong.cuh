@@ -601,6 +601,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         ScoreConsts sc = {};
         if constexpr (SCORE != kScorePlain) sc = make_score_consts(p.scale, p.softcap, it.slope[qt]);
         const int niter = tr.jhi - tr.jlo;
+        const bool relu_raw = RELU && p.softcap == 0.f && it.slope[qt] == 0.f && p.scale > 0.f;
         CapPoly poly = {};                                   // softcap: coefficients of a tile's second pass
         float m_used = -INFINITY, l = 0.f;
         // Bias-only score (Appendix A.1): s*scale + slope*(i' - j) in log2 units = s*cs + slope2*(rowoff_chunk - i).
@@ -664,7 +665,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                             y[c * 32 + 2 * k2 + 1] = __float_as_uint(s1);
                         }
                     } else if constexpr (SCORE != kScorePlain) {
-                        if constexpr (SIGMOID || RELU) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                        if constexpr (SIGMOID || RELU) {
+                            // (ReLU of a plainly scaled score: max(scale * s, 0) = scale * max(s, 0) for scale > 0, so
+                            // the raw scores go on and the scale joins the epilogue's factor.)
+                            if (!(RELU && relu_raw)) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                        }
                         else if constexpr (kRedo) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
                         else score_chunk32_quad(&y[c * 32], sc, rowoff - (float)(c * 32), zmax);
                     }
@@ -801,7 +806,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             if (!bounded_wait(ptx::smem_u32(&bars->pv_done[qt]), (g - 1u) & 1u, bars, p.status_word)) return;
             ptx::tc_fence_after_sync();
         }
-        const float inv = SIGMOID ? p.out_scale : (RELU ? p.out_scale * kLn2 : (l > 0.f ? 1.0f / l : 0.f));
+        const float inv = SIGMOID ? p.out_scale : (RELU ? (relu_raw ? p.out_scale * p.scale : p.out_scale * kLn2) : (l > 0.f ? 1.0f / l : 0.f));
         char* obase = reinterpret_cast<char*>(p.o) +
                       ((long long)it.b * p.os[0] + (long long)it.ht[qt] * p.os[1] + (long long)row * p.os[2]) * (p.o_fp32 ? 4 : 2);
 #pragma unroll 1
