@@ -574,8 +574,11 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
 #pragma unroll
             for (int c = 0; c < kWgCols / 32; ++c) {
                 if constexpr (SCORE != kScorePlain && !kTileCap) {
-                    // (Sigmoid without softcap or bias: the scale rides in the sigmoid's own first FMA, below.)
-                    if (!(SIGMOID && !sc.softcap && !sc.has_bias)) score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                    // (Sigmoid without softcap or bias: the scale rides in the sigmoid's own first FMA, below.  ReLU of a
+                    // plainly scaled score: max(scale * s, 0) = scale * max(s, 0) for scale > 0, so the raw scores go
+                    // on and the scale joins the epilogue's factor.)
+                    if (!((SIGMOID || (RELU && p.scale > 0.f)) && !sc.softcap && !sc.has_bias))
+                        score_chunk32<SCORE == kScoreGeneric>(&y[c * 32], sc, rowoff - (float)(c * 32));
                 }
                 if (!full_tile) mask_chunk32_cmp(&y[c * 32], mask_a - c * 32, mask_e - c * 32);   // (the bit-test form cost this kernel 2 %)
                 if (!SIGMOID && !RELU && !fixed_max) {
@@ -724,7 +727,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             ++items_done;
             ptx::tc_fence_after_sync();
         }
-        const float inv = SIGMOID ? p.out_scale * 0.0009765625f : (RELU ? p.out_scale * kLn2 : (l_row > 0.f ? 1.0f / l_row : 0.f));
+        const bool relu_raw = RELU && p.scale > 0.f && !sc.softcap && !sc.has_bias;       // P holds max(s, 0) of the raw scores
+        const float inv = SIGMOID ? p.out_scale * 0.0009765625f
+                                  : (RELU ? (relu_raw ? p.out_scale * p.scale : p.out_scale * kLn2) : (l_row > 0.f ? 1.0f / l_row : 0.f));
         char* obase = reinterpret_cast<char*>(p.o) +
                       ((long long)it.b * p.os[0] + (long long)it.h * p.os[1] + (long long)row * p.os[2] + wg * kOC) * (p.o_fp32 ? 4 : 2);
 #pragma unroll
