@@ -602,6 +602,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         if constexpr (SCORE != kScorePlain) sc = make_score_consts(p.scale, p.softcap, it.slope[qt]);
         const int niter = tr.jhi - tr.jlo;
         const bool relu_raw = RELU && p.softcap == 0.f && it.slope[qt] == 0.f && p.scale > 0.f;
+        const bool sig_raw = SIGMOID && p.softcap == 0.f && it.slope[qt] == 0.f;
         CapPoly poly = {};                                   // softcap: coefficients of a tile's second pass
         float m_used = -INFINITY, l = 0.f;
         // Bias-only score (Appendix A.1): s*scale + slope*(i' - j) in log2 units = s*cs + slope2*(rowoff_chunk - i).
@@ -668,7 +669,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                         if constexpr (SIGMOID || RELU) {
                             // (ReLU of a plainly scaled score: max(scale * s, 0) = scale * max(s, 0) for scale > 0, so
                             // the raw scores go on and the scale joins the epilogue's factor.)
-                            if (!(RELU && relu_raw)) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
+                            // (Sigmoid of a plainly scaled score: the scale rides in the sigmoid's first FMA, below.)
+                            if (!((RELU && relu_raw) || (SIGMOID && sig_raw))) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
                         }
                         else if constexpr (kRedo) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
                         else score_chunk32_quad(&y[c * 32], sc, rowoff - (float)(c * 32), zmax);
@@ -723,7 +725,8 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 // be carried by a few large weights, so bf16 rounding of P (up to 2^-8 relative) would show in O: P is split into
                 // P_hi = bf16(p) in columns [0,64) and the residual P_lo = bf16(p - P_hi) in columns [64,128) of the
                 // S buffer; the MMA thread accumulates both.  out_scale is applied in the epilogue.
-                const uint64_t nb2 = ptx::pack2(-sig_bias2, -sig_bias2), neg1 = ptx::pack2(-1.0f, -1.0f);
+                const float neg_mul = sig_raw ? -sc.cs : -1.0f;     // raw scores in, or scores in log2 units
+                const uint64_t nb2 = ptx::pack2(-sig_bias2, -sig_bias2), neg1 = ptx::pack2(neg_mul, neg_mul);
 #pragma unroll
                 for (int cc = 0; cc < kBN / 32; ++cc) {
                     uint32_t pk[16], pl[16];
