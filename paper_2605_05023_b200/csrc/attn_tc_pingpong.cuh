@@ -812,60 +812,33 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
         const float inv = SIGMOID ? p.out_scale : (RELU ? (relu_raw ? p.out_scale * p.scale : p.out_scale * kLn2) : (l > 0.f ? 1.0f / l : 0.f));
         char* obase = reinterpret_cast<char*>(p.o) +
                       ((long long)it.b * p.os[0] + (long long)it.ht[qt] * p.os[1] + (long long)row * p.os[2]) * (p.o_fp32 ? 4 : 2);
-#pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t orr[32];
+        if constexpr (TMA_OUT) {
+            // bf16 output, two heads x 128 rows per item (both tiles end together and their epilogues compete for
+            // the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
+            // in shared memory (64-byte swizzle: the 16-byte piece k of row r sits at piece k ^ ((r >> 1) & 3),
+            // conflict free) and leave as one TMA tile store, which also clips rows beyond Sq.  A thread-owns-a-row
+            // store to global memory touches 32 lines per instruction; this way the stores cost the load/store
+            // unit an eighth of that.  The whole accumulator row is read first: one wait covers all the loads, and
+            // the next item's first P V may overwrite the accumulator that much earlier.
+            uint32_t oall[D / 32][32];
             if (niter > 0) {
-                ptx::tmem_ld_32x32(tm + ocol + c * 32, orr);
-                ptx::tmem_wait_ld_regs(orr);
-                if (c == D / 32 - 1) {
-                    // All of O is in registers: the next item's first P V may overwrite the accumulator.
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->o_free[qt]));
-                }
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) ptx::tmem_ld_32x32(tm + ocol + c * 32, oall[c]);
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) ptx::tmem_wait_ld_regs(oall[c]);
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->o_free[qt]));
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) orr[i] = 0u;
+                for (int c = 0; c < D / 32; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) oall[c][i] = 0u;
             }
-            if (p.o_fp32) {
-                if (store_row) {
-                    float4* dst = reinterpret_cast<float4*>(obase + c * 128);
+            const int r = threadIdx.x & 31;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[i] = make_float4(__uint_as_float(orr[4 * i]) * inv, __uint_as_float(orr[4 * i + 1]) * inv,
-                                             __uint_as_float(orr[4 * i + 2]) * inv, __uint_as_float(orr[4 * i + 3]) * inv);
-                }
-            } else if constexpr (!TMA_OUT) {
-                // bf16 output, 256 consecutive rows per item: under a causal mask the first tile's epilogue runs under the
-                // second tile's last key step, and the threads go on at once, so plain stores by the row's owner are best:
-                // 32 bytes at a time (a whole sector per thread and instruction; with 16-byte stores the exposed epilogue
-                // of the second tile took 3.7 k cycles, nearly all of them in the load/store unit).
-                if (store_row) {
-                    char* dst = obase + c * 64;
-                    const bool aligned32 = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;     // (always, for dense rows)
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        uint32_t w[8];
-#pragma unroll
-                        for (int k2 = 0; k2 < 8; ++k2)
-                            w[k2] = ptx::pack_bf16x2(__uint_as_float(orr[16 * i + 2 * k2]) * inv, __uint_as_float(orr[16 * i + 2 * k2 + 1]) * inv);
-                        if (aligned32) {
-                            ptx::st_global_v8(dst + i * 32, w);
-                        } else {
-                            reinterpret_cast<uint4*>(dst + i * 32)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                            reinterpret_cast<uint4*>(dst + i * 32)[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                        }
-                    }
-                }
-            } else {
-                // bf16 output, two heads x 128 rows per item (both tiles end together and their epilogues compete for
-                // the load/store unit): the warp's 32 rows x 32 columns go through one of its own two 2 KB boxes
-                // in shared memory (64-byte swizzle: the 16-byte piece k of row r sits at piece k ^ ((r >> 1) & 3),
-                // conflict free) and leave as one TMA tile store, which also clips rows beyond Sq.  A thread-owns-a-row
-                // store to global memory touches 32 lines per instruction; this way the stores cost the load/store
-                // unit an eighth of that.
-                const int r = threadIdx.x & 31;
+            for (int c = 0; c < D / 32; ++c) {
+                const uint32_t (&orr)[32] = oall[c];
                 if (r == 0) ptx::bulk_wait_group_read1();        // the store before last has been read out of its box
                 __syncwarp();
                 uint4* dst = reinterpret_cast<uint4*>(stage_ptr + (c & 1) * C::kStageBytes + r * 64);
@@ -883,6 +856,55 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                 if (r == 0) {
                     ptx::tma_store_4d(tmap_o, stage_smem + (c & 1) * C::kStageBytes, c * 32, q0 + (wg_thread & ~31), it.ht[qt], it.b);
                     ptx::bulk_commit_group();
+                }
+            }
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t orr[32];
+                if (niter > 0) {
+                    ptx::tmem_ld_32x32(tm + ocol + c * 32, orr);
+                    ptx::tmem_wait_ld_regs(orr);
+                    if (c == D / 32 - 1) {
+                        // All of O is in registers: the next item's first P V may overwrite the accumulator.
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(ptx::smem_u32(&bars->o_free[qt]));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) orr[i] = 0u;
+                }
+                if (p.o_fp32) {
+                    if (store_row) {
+                        float4* dst = reinterpret_cast<float4*>(obase + c * 128);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_float4(__uint_as_float(orr[4 * i]) * inv, __uint_as_float(orr[4 * i + 1]) * inv,
+                                                 __uint_as_float(orr[4 * i + 2]) * inv, __uint_as_float(orr[4 * i + 3]) * inv);
+                    }
+                } else {
+                    // bf16 output, 256 consecutive rows per item: under a causal mask the first tile's epilogue runs under the
+                    // second tile's last key step, and the threads go on at once, so plain stores by the row's owner are best:
+                    // 32 bytes at a time (a whole sector per thread and instruction; with 16-byte stores the exposed epilogue
+                    // of the second tile took 3.7 k cycles, nearly all of them in the load/store unit).
+                    if (store_row) {
+                        char* dst = obase + c * 64;
+                        const bool aligned32 = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;     // (always, for dense rows)
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            uint32_t w[8];
+#pragma unroll
+                            for (int k2 = 0; k2 < 8; ++k2)
+                                w[k2] = ptx::pack_bf16x2(__uint_as_float(orr[16 * i + 2 * k2]) * inv, __uint_as_float(orr[16 * i + 2 * k2 + 1]) * inv);
+                            if (aligned32) {
+                                ptx::st_global_v8(dst + i * 32, w);
+                            } else {
+                                reinterpret_cast<uint4*>(dst + i * 32)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                                reinterpret_cast<uint4*>(dst + i * 32)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                            }
+                        }
+                    }
                 }
             }
         }
