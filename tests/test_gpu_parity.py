@@ -415,7 +415,7 @@ import os, sys
 sys.path.insert(0, sys.argv[1]); sys.path.insert(0, os.path.join(sys.argv[1], "tests"))
 import test_gpu_parity as t
 from synth_inputs import small_workloads
-for w in small_workloads() + t.BF16_EXTRA:
+for w in small_workloads() + t.BF16_EXTRA + [w for w in t.random_combinations(96, 20261125) if w.dtype == "bf16"]:
     t.check(w)
 # many short work items per CTA (the ring wraps, work items are handed out by the hardware) on the forced kernel
 import torch, paper_2605_05023_b200 as pk
@@ -568,6 +568,90 @@ LONG_CASES = [
 @pytest.mark.parametrize("w", LONG_CASES, ids=lambda w: w.name)
 def test_long_sequences_sampled_rows(w):
     check(w, rows=sampled_rows(w, 24, 1, seed=sum(map(ord, w.name)), every_head=8))
+
+
+# ------------------------------------------------------------------ seeded random combinations
+# The cases above pick their combinations by hand.  Here shape, GQA group, mask clauses, score modifiers and normaliser
+# are drawn together from one seeded generator, so that combinations nobody thought of (a ragged Sq != Sk under a
+# two-sided window with a bias and fp32 output, a test query over global tokens, ...) meet the oracle too.  Every
+# case of the first set is small enough for the full oracle; the second set (``large``: bf16, 1200 to 4500 tokens,
+# grids of several hundred work items, so that the work order, the deferred blocks and the ring wrap-around take
+# part) is compared on sampled rows.
+def random_combinations(n, seed, large=False):
+    rng = np.random.RandomState(seed)
+    out = []
+    for idx in range(n):
+        fp32 = (not large) and rng.rand() < 0.15
+        D = int(rng.choice([16, 32, 64, 128, 256])) if fp32 else int(rng.choice([64, 128, 128, 256]))
+        hkv = int(rng.choice([1, 2, 4] if large else [1, 2]))
+        group = int(rng.choice([1, 1, 2, 4, 8] if large else [1, 1, 2, 3, 4, 8]))
+        B = int(rng.choice([1, 2, 3] if large else [1, 2]))
+        smin = 1200 if large else 1
+        smax = 4500 if large else 300 if fp32 else (420 if D == 256 else 640)
+        wide = [127, 511, 1024] if large else []
+        sq = int(rng.randint(smin, smax + 1))
+        sk = sq if rng.rand() < 0.6 else int(rng.randint(smin, smax + 1))
+        kw = {}
+        mask = rng.choice(["none", "causal", "causal_window", "window", "docs", "docs_bidir", "prefix", "prefix_window",
+                           "global_window", "share_question", "test_query"])
+        if mask in ("docs", "docs_bidir", "share_question", "test_query"):
+            B, sk = 1, sq
+            cuts = sorted(set(int(c) for c in rng.randint(0, sq + 1, size=int(rng.randint(1, 9 if large else 6)))) | {0, sq})
+            if rng.rand() < 0.5 and len(cuts) > 2:
+                cuts = cuts[:2] + [cuts[1]] + cuts[2:]          # an empty document
+            kw["cu_seqlens"] = tuple(cuts)
+            kw["causal"] = mask != "docs_bidir"
+            if mask == "share_question":
+                kw["global_len"] = int(cuts[1])
+            if mask == "test_query":
+                kw["test_query_start"] = int(rng.randint(0, sq + 1))
+        elif mask == "causal":
+            kw["causal"] = True
+        elif mask == "causal_window":
+            kw.update(causal=True, window_left=int(rng.choice([0, 1, 31, 127, 128, 300] + wide)), window_right=0)
+        elif mask == "window":
+            kw.update(window_left=int(rng.choice([0, 5, 64, 200] + wide)), window_right=int(rng.choice([0, 5, 64, 200] + wide)))
+        elif mask == "prefix":
+            kw.update(causal=True, prefix_len=int(rng.randint(0, sk + 1)))
+        elif mask == "prefix_window":
+            kw.update(causal=True, prefix_len=int(rng.randint(0, sk + 1)), window_left=int(rng.choice([3, 40, 150] + wide)), window_right=0)
+        elif mask == "global_window":
+            kw.update(window_left=int(rng.choice([2, 30, 130] + wide)), window_right=int(rng.choice([0, 30, 130] + wide)),
+                      global_len=int(rng.randint(0, min(sk, 200) + 1)), causal=bool(rng.rand() < 0.4))
+        norm = rng.choice(["softmax", "softmax", "softmax", "softmax", "sigmoid", "relu"])
+        if norm == "sigmoid":
+            kw.update(normalizer="sigmoid", sigmoid_bias=-math.log(float(sk)))
+        elif norm == "relu":
+            kw.update(normalizer="relu", out_scale=1.0 / sk)
+        score = rng.choice(["none", "none", "softcap", "bias", "both"])
+        hq = hkv * group
+        if score in ("softcap", "both"):
+            kw["softcap"] = float(rng.choice([1.0, 5.0, 30.0, 50.0]))
+        if score in ("bias", "both"):
+            kind = rng.choice(["alibi", "plus_one", "mixed"])
+            kw["slopes"] = (alibi_slopes(hq) if kind == "alibi" else tuple([1.0] * hq) if kind == "plus_one"
+                            else tuple(float(x) for x in rng.uniform(-0.5, 0.5, size=hq)))
+        if rng.rand() < 0.25:
+            kw["scale"] = float(rng.choice([0.05, 0.2, 1.0 / math.sqrt(D) * 1.7]))
+        o_dtype = "fp32" if fp32 or rng.rand() < 0.3 else "bf16"
+        std = float(rng.choice([1.0, 1.5]))
+        # The sigmoid normaliser does not normalise rows: with wide inputs or a growing bias |O| passes 5.12, from
+        # where on half a bf16 spacing alone exceeds the bound on O; such cases store fp32, as configuration 4(b) does.
+        if norm == "sigmoid" and (std > 1.0 or "slopes" in kw):
+            o_dtype = "fp32"
+        out.append(Workload(f"{'R' if large else 'r'}{idx:02d}_{mask}_{norm}_{score}_d{D}_g{group}", B, hq, hkv, sq, sk, D,
+                            dtype="fp32" if fp32 else "bf16", o_dtype=o_dtype, std=std, seed=3000 + idx, **kw))
+    return out
+
+
+@pytest.mark.parametrize("w", random_combinations(96, 20261125), ids=lambda w: w.name)
+def test_seeded_random_combinations(w):
+    check(w)
+
+
+@pytest.mark.parametrize("w", random_combinations(32, 20261126, large=True), ids=lambda w: w.name)
+def test_seeded_random_combinations_of_many_work_items(w):
+    check(w, rows=sampled_rows(w, 24, 2, seed=sum(map(ord, w.name)), every_head=6))
 
 
 # ------------------------------------------------------------------ masked positions have no influence (on the GPU)
