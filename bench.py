@@ -51,8 +51,8 @@ STEP_SETS = {
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of one launch); a step set reports the mean
 # over its launches; None where no capture exists.
 NCU_TRAFFIC_BYTES_PER_VARIANT = {
-    "c2_noncausal": 318.6e6, "c2_causal": 339.5e6, "c3_gqa_window_alibi": 308.7e6,
-    "c4a_softcap": 346.2e6, "c4b_sigmoid": 409.1e6, "c5_packed_doc_causal": 1152.1e6,
+    "c2_noncausal": 314.3e6, "c2_causal": 344.6e6, "c3_gqa_window_alibi": 309.9e6,
+    "c4a_softcap": 344.3e6, "c4b_sigmoid": 395.2e6, "c5_packed_doc_causal": 1157.4e6,
 }
 
 
