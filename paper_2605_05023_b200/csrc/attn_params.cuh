@@ -42,6 +42,7 @@ struct AttnParams {
     int global_len;             // global tokens: positions < global_len pass the window / document clauses (0 = none)
     int head_pair;              // ping-pong kernel: a work item is two heads x 128 rows (1) or one head x 256 rows (0)
     int defer_blocks;           // tensor-core kernels: query blocks per head whose work items end the work order (see work_order)
+    int front_blocks;           // ... and whose work items open it (see leading_blocks)
 };
 
 struct RowInterval {
@@ -159,7 +160,43 @@ __device__ __forceinline__ void work_order(int lin, int units_total, int sec_uni
     }
 }
 
+// The same with `front` blocks per unit that open the work order, before all sections, block by block over all units
+// (rank < front): the blocks that hold the rows of global tokens under a non-causal mask, whose items walk every
+// key tile while the others walk a window (see leading_blocks).  Every (rank, unit) pair still has exactly one index.
+__device__ __forceinline__ void work_order_front(int lin, int units_total, int sec_units, int nqb, int defer, int front,
+                                                 int& rank, int& unit) {
+    const int front_items = units_total * front;
+    if (lin < front_items) {
+        rank = lin / units_total;
+        unit = lin - rank * units_total;
+    } else {
+        work_order(lin - front_items, units_total, sec_units, nqb - front, defer, rank, unit);
+        rank += front;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ host side
+// How many query blocks of every head hold a global token's row under a non-causal two-sided window (Global Sliding
+// Window, Appendix A.2): such a row sees every key, so its block's work item is the longest of its head by far, and
+// handed out section by section the last section's long items can end the grid on a few SMs.  They open the work
+// order instead, when that helps: 0 under a causal mask (it bounds those rows like the others), without global
+// tokens, when the long items have fewer than four times the key tiles of the window items, when a section lasts
+// longer than a long item anyway (then the long items of the last section are hidden in it, and section order keeps
+// its K and V in L2), or when more than a quarter of the blocks would qualify.  `sec_units`: work-order units
+// ((batch, head) or head pairs) per section; `workers`: CTAs that run at once.
+inline int leading_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long sec_units, int workers) {
+    if (!(p.mask_flags & kMaskGlobal) || (p.mask_flags & kMaskCausal) || nqb < 4) return 0;
+    if (!(p.mask_flags & kMaskWindow) || p.window_left < 0 || p.window_right < 0) return 0;
+    const long long window_tiles = ((long long)p.window_left + p.window_right + rows) / key_tile + 2;
+    const long long long_tiles = (long long)p.Sk / key_tile;
+    if (long_tiles < 4 * window_tiles) return 0;
+    const long long global_rows = std::min<long long>(std::max<long long>((long long)p.global_len - (p.Sk - p.Sq), 0), p.Sq);
+    const int blocks = (int)((global_rows + rows - 1) / rows);
+    if (blocks * 4 > nqb) return 0;
+    const long long section_steps = sec_units * (blocks * long_tiles + (nqb - blocks) * window_tiles) / std::max(workers, 1);
+    return (section_steps >= long_tiles) ? 0 : blocks;
+}
+
 // How many of the first (lightest) query blocks of every head go to the end of the work order (decode_item of the
 // ping-pong and of the CTA-pair kernel).  Causal masks without documents or global tokens only: there a block's key
 // tiles grow with its index, and the count follows from the row intervals.  `rows`: query rows of a work item;

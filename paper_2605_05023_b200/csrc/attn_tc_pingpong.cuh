@@ -157,7 +157,7 @@ __device__ __forceinline__ TileRange tile_range(const AttnParams& p, int q0, int
 // block first, the lightest blocks of every head at the very end).  `order`, when not null, lists the query blocks of
 // a head heaviest first (packed documents, see build_block_order); otherwise the blocks are taken from the last to
 // the first (most keys under a causal mask).
-template <int NQ>
+template <int NQ, bool GLB>
 __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const uint16_t* order) {
     // The two query tiles of an item share every K / V tile.  With an even GQA group they are the same 128 rows
     // of two neighbouring query heads of one KV group (identical key ranges: no step in which only one of them
@@ -170,7 +170,9 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     const int bh_total = p.B * p.Hq / units;
     const int sec_units = p.sec_heads / units;
     int rank, bh;                                        // rank of the block among its head's blocks, heaviest first
-    work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh);
+    // (only masks with global tokens have leading blocks; the other instances keep the plain order's code)
+    if constexpr (GLB) work_order_front(lin, bh_total, sec_units, nqb, p.defer_blocks, p.front_blocks, rank, bh);
+    else work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh);
     const int qb = order ? (int)order[rank] : nqb - 1 - rank;
     const int hq_units = p.Hq / units;
     ItemG it;
@@ -295,7 +297,7 @@ __device__ __forceinline__ bool next_item(Barriers* bars, uint32_t& phase, int32
 // following ones are CTAs of the grid that have not started, taken over with cluster launch control (clc_fetch:
 // only this thread touches the hardware scheduler's response).  It publishes {handed over, decoded item} with
 // ordinary stores for the other roles, so that no role spends time on index arithmetic and mask intervals.
-template <int NQ>
+template <int NQ, bool GLB>
 __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* bars, int order_capacity) {
     // the heaviest-first order of the query blocks sits right behind the barrier block (see build_block_order)
     const uint16_t* order = has_block_order<NQ>(p, order_capacity) ? reinterpret_cast<const uint16_t*>(reinterpret_cast<const uint8_t*>(bars) + 1024) : nullptr;
@@ -305,7 +307,7 @@ __device__ __forceinline__ void scheduler_role(const AttnParams& p, Barriers* ba
         volatile int* m = bars->item_msg;
         m[0] = got ? 1 : 0;
         if (got) {
-            const ItemG it = decode_item<NQ>(p, lin, order);
+            const ItemG it = decode_item<NQ, GLB>(p, lin, order);
             m[1] = it.q0t[0]; m[2] = it.q0t[1]; m[3] = it.ht[0]; m[4] = it.ht[1]; m[17] = it.b; m[18] = it.g;
             m[5] = it.tr[0].jlo; m[6] = it.tr[0].jhi; m[7] = it.tr[1].jlo; m[8] = it.tr[1].jhi;
             m[9] = it.lo_max[0]; m[10] = it.hi_min[0]; m[11] = it.lo_max[1]; m[12] = it.hi_min[1];
@@ -982,7 +984,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
         } else if (warp == C::kMmaWarp) {
             if (lane == 0) mma_role<D, NQ, NORM == kNormSigmoid>(p, bars, tmem, q_smem, ring_smem);
         } else if (warp == C::kSchedWarp) {
-            if (lane == 0) scheduler_role<NQ>(p, bars, C::kMaxOrdered);
+            if (lane == 0) scheduler_role<NQ, GLB>(p, bars, C::kMaxOrdered);
         } else if (blockIdx.x == 0 && (p.mask_flags & kMaskDocument)) {
             check_offsets_warp(p.cu, p.num_docs, p.Sq, p.status_word);     // the spare warp of the first CTA
         }
@@ -1034,6 +1036,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     const long long grid = nqb * (bh / (p.head_pair ? 2 : 1));
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
     p.defer_blocks = deferred_blocks(p, (int)rows, kBN, (int)nqb, bh / (p.head_pair ? 2 : 1), device_sm_count());
+    // (the blocks of global tokens' rows are the first of the weight-ordered list, which needs its table)
+    p.front_blocks = (GLB && nqb <= C::kMaxOrdered) ? leading_blocks(p, (int)rows, kBN, (int)nqb, sec / (p.head_pair ? 2 : 1), device_sm_count()) : 0;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }

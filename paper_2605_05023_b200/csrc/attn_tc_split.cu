@@ -119,8 +119,9 @@ __device__ __forceinline__ Item decode_item(const AttnParams& p, int lin) {
     const int nqb = (p.Sq + kBM - 1) / kBM;
     const int bh_total = p.B * p.Hq;
     int rank, bh;
-    work_order(lin, bh_total, p.sec_heads, nqb, 0, rank, bh);      // (this kernel defers no blocks)
-    const int qb = nqb - 1 - rank;
+    work_order_front(lin, bh_total, p.sec_heads, nqb, 0, p.front_blocks, rank, bh);      // (this kernel defers no blocks)
+    // the first blocks (rows of global tokens under a non-causal mask) open the order, the others run from the last down
+    const int qb = rank < p.front_blocks ? rank : nqb - 1 - (rank - p.front_blocks);
     Item it;
     it.b = bh / p.Hq;
     it.h = bh - it.b * p.Hq;
@@ -726,6 +727,7 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     const long long nqb = (p.Sq + kBM - 1) / kBM;
     const long long grid = nqb * bh;
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
+    p.front_blocks = leading_blocks(p, kBM, kBN, (int)nqb, sec, device_sm_count());
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }

@@ -173,6 +173,13 @@ BF16_EXTRA = [
     Workload("b_global_sq_lt_sk", 1, 1, 1, 300, 800, 128, seed=67, causal=True, window_left=50, window_right=0, global_len=140),
     Workload("b_global_relu", 1, 2, 2, 700, 700, 128, seed=68, window_left=64, window_right=64, global_len=200,
              normalizer="relu", out_scale=1.0 / 700.0),
+    # the blocks that hold global tokens' rows open the work order (non-causal, narrow window, at least 16 key tiles;
+    # one and two such blocks per head; 256-row items, two-head items, D = 256; Sq != Sk shifts which rows are global)
+    Workload("b_global_front_1", 2, 3, 3, 2200, 2200, 128, seed=140, window_left=10, window_right=10, global_len=100),
+    Workload("b_global_front_2_pair", 2, 4, 2, 2100, 2100, 64, seed=141, window_left=10, window_right=5, global_len=200),
+    Workload("b_global_front_d256", 1, 2, 1, 1600, 1600, 256, seed=142, window_left=5, window_right=5, global_len=150, std=1.5),
+    Workload("b_global_front_sq_lt_sk", 1, 2, 2, 1800, 2300, 128, seed=143, window_left=10, window_right=10, global_len=700),
+    Workload("b_global_front_sq_gt_sk", 1, 2, 1, 2000, 1800, 128, seed=144, window_left=10, window_right=10, global_len=20),
     Workload("b_share_question_1k", 1, 2, 2, 1024, 1024, 128, seed=69, causal=True,
              cu_seqlens=(0, 300, 301, 512, 640, 1000, 1024), global_len=300),
     Workload("b_share_question_sigmoid", 1, 1, 1, 640, 640, 128, seed=70, causal=True, cu_seqlens=(0, 128, 384, 640),
