@@ -43,6 +43,7 @@ struct AttnParams {
     int head_pair;              // ping-pong kernel: a work item is two heads x 128 rows (1) or one head x 256 rows (0)
     int defer_blocks;           // tensor-core kernels: query blocks per head whose work items end the work order (see work_order)
     int front_blocks;           // ... and whose work items open it (see leading_blocks)
+    int sec_merge_from;         // ping-pong kernel: the sections from this one on are handed out as one (see work_order)
 };
 
 struct RowInterval {
@@ -143,14 +144,18 @@ __device__ __forceinline__ TileBounds tile_bounds(const AttnParams& p, int q0, i
 // coordinate and runs from the heaviest block of a unit (rank 0) to the lightest, so the hardware hands out the
 // heaviest items first.  The `defer` lightest blocks of every unit come after all sections, again heaviest first
 // (see deferred_blocks).  rank: position of the block among its unit's `nqb` blocks, heaviest first.
-__device__ __forceinline__ void work_order(int lin, int units_total, int sec_units, int nqb, int defer, int& rank, int& unit) {
+// The sections from `merge_from` on form one section: a last section that holds less work per SM than its longest
+// item takes ends the grid with idle SMs; as part of a longer section its long items start earlier and its light
+// ones fill the end.
+__device__ __forceinline__ void work_order(int lin, int units_total, int sec_units, int nqb, int defer, int& rank, int& unit,
+                                           int merge_from = 0x7fffffff) {
     const int nh = nqb - defer;                          // blocks per unit that are taken section by section
     if (lin < units_total * nh) {
         const int per_sec = sec_units * nh;
-        const int sec = lin / per_sec;
+        const int sec = min(lin / per_sec, merge_from);
         const int r = lin - sec * per_sec;
         const int sec_start = sec * sec_units;
-        const int sh = min(sec_units, units_total - sec_start);
+        const int sh = min(sec >= merge_from ? units_total : sec_units, units_total - sec_start);
         rank = r / sh;
         unit = sec_start + r % sh;
     } else {                                             // the deferred blocks: one last section of all units

@@ -172,7 +172,7 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     int rank, bh;                                        // rank of the block among its head's blocks, heaviest first
     // (only masks with global tokens have leading blocks; the other instances keep the plain order's code)
     if constexpr (GLB) work_order_front(lin, bh_total, sec_units, nqb, p.defer_blocks, p.front_blocks, rank, bh);
-    else work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh);
+    else work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh, p.sec_merge_from);
     const int qb = order ? (int)order[rank] : nqb - 1 - rank;
     const int hq_units = p.Hq / units;
     ItemG it;
@@ -1037,6 +1037,13 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
     p.defer_blocks = deferred_blocks(p, (int)rows, kBN, (int)nqb, bh / (p.head_pair ? 2 : 1), device_sm_count());
     // (the blocks of global tokens' rows are the first of the weight-ordered list, which needs its table)
+    // Packed documents: a section is one or a few heads, and its longest items (a document's last blocks) can take
+    // longer than an SM's share of the section, so the last two sections are handed out as one.
+    {
+        const long long sec_units = sec / (p.head_pair ? 2 : 1), units = bh / (p.head_pair ? 2 : 1);
+        const long long sections = (units + sec_units - 1) / sec_units;
+        p.sec_merge_from = ((p.mask_flags & kMaskDocument) && sections >= 2) ? (int)(sections - 2) : 0x7fffffff;
+    }
     p.front_blocks = (GLB && nqb <= C::kMaxOrdered) ? leading_blocks(p, (int)rows, kBN, (int)nqb, sec / (p.head_pair ? 2 : 1), device_sm_count()) : 0;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
