@@ -169,13 +169,13 @@ __device__ __forceinline__ void work_order(int lin, int units_total, int sec_uni
 // (rank < front): the blocks that hold the rows of global tokens under a non-causal mask, whose items walk every
 // key tile while the others walk a window (see leading_blocks).  Every (rank, unit) pair still has exactly one index.
 __device__ __forceinline__ void work_order_front(int lin, int units_total, int sec_units, int nqb, int defer, int front,
-                                                 int& rank, int& unit) {
+                                                 int& rank, int& unit, int merge_from = 0x7fffffff) {
     const int front_items = units_total * front;
     if (lin < front_items) {
         rank = lin / units_total;
         unit = lin - rank * units_total;
     } else {
-        work_order(lin - front_items, units_total, sec_units, nqb - front, defer, rank, unit);
+        work_order(lin - front_items, units_total, sec_units, nqb - front, defer, rank, unit, merge_from);
         rank += front;
     }
 }

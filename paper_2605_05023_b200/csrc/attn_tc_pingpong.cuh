@@ -171,7 +171,7 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     const int sec_units = p.sec_heads / units;
     int rank, bh;                                        // rank of the block among its head's blocks, heaviest first
     // (only masks with global tokens have leading blocks; the other instances keep the plain order's code)
-    if constexpr (GLB) work_order_front(lin, bh_total, sec_units, nqb, p.defer_blocks, p.front_blocks, rank, bh);
+    if constexpr (GLB) work_order_front(lin, bh_total, sec_units, nqb, p.defer_blocks, p.front_blocks, rank, bh, p.sec_merge_from);
     else work_order(lin, bh_total, sec_units, nqb, p.defer_blocks, rank, bh, p.sec_merge_from);
     const int qb = order ? (int)order[rank] : nqb - 1 - rank;
     const int hq_units = p.Hq / units;
@@ -251,12 +251,18 @@ __device__ __noinline__ void build_block_order(const AttnParams& p, uint16_t* or
     const int nqb = (p.Sq + rows - 1) / rows;
     if (!has_block_order<NQ>(p, capacity)) return;
     for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
-        int jlo = 0x7fffffff, jhi = 0;
+        // key tiles of the block's work item, as decode_item counts them: the window / document tiles [jlo, jhi) and,
+        // in front of them, the tiles [0, pend) of the global tokens (the prompt of a Share Question mask is most of
+        // an item's keys)
+        int jlo = 0x7fffffff, jhi = 0, pend = 0;
         for (int t = 0; t < (p.head_pair ? 1 : NQ); ++t) {
             const TileBounds tb = tile_bounds(p, qb * rows + t * kBM, kBM);
-            if (tb.any && tb.hi_max >= 0 && tb.lo_min <= tb.hi_max) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
+            if (!tb.any) continue;
+            pend = max(pend, (tb.pre_max + kBN - 1) / kBN);
+            if (tb.hi_max >= 0 && tb.lo_min <= tb.hi_max) { jlo = min(jlo, tb.lo_min / kBN); jhi = max(jhi, tb.hi_max / kBN + 1); }
         }
-        weight[qb] = (uint16_t)min(max(jhi - jlo, 0), 65535);      // (the few tiles of global keys in front are not counted)
+        const int tiles = (jlo >= jhi) ? pend : (jlo <= pend ? max(jhi, pend) : pend + (jhi - jlo));
+        weight[qb] = (uint16_t)min(tiles, 65535);
     }
     __syncthreads();
     for (int qb = threadIdx.x; qb < nqb; qb += blockDim.x) {
