@@ -52,7 +52,7 @@ STEP_SETS = {
 # over its launches; None where no capture exists.
 NCU_TRAFFIC_BYTES_PER_VARIANT = {
     "c2_noncausal": 314.3e6, "c2_causal": 344.6e6, "c3_gqa_window_alibi": 309.9e6,
-    "c4a_softcap": 344.3e6, "c4b_sigmoid": 395.2e6, "c5_packed_doc_causal": 1157.4e6,
+    "c4a_softcap": 344.3e6, "c4b_sigmoid": 395.2e6, "c5_packed_doc_causal": 1182.3e6,
 }
 
 
