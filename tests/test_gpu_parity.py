@@ -71,6 +71,10 @@ def check(w, rows=None):
         if rows is None:
             ratio = np.abs(o_np - o_ref) / relu_row_bounds(w, v, o_ref, p_ref)
             assert ratio.max() <= 1.0, f"{w.name}: per-row ReLU bound exceeded {ratio.max():.2f} times"
+    if w.normalizer == "sigmoid" and w.dtype == "fp32":
+        # no row normalisation either: |O| grows with the number of keys whose weight is near 1, and fp32 rounding
+        # (1e-7 relative per step) with it; the fp32 bound is relative to the largest output once that passes 1.
+        tol_o = tol_o * max(1.0, float(np.abs(o_ref).max()))
     err_o = np.abs(o_np - o_ref).max()
     assert err_o <= tol_o, f"{w.name}: max|dO| = {err_o:.3e} > {tol_o}"
     if l_np is not None:
@@ -422,8 +426,11 @@ import os, sys
 sys.path.insert(0, sys.argv[1]); sys.path.insert(0, os.path.join(sys.argv[1], "tests"))
 import test_gpu_parity as t
 from synth_inputs import small_workloads
-for w in small_workloads() + t.BF16_EXTRA + [w for w in t.random_combinations(96, 20261125) if w.dtype == "bf16"]:
+for w in small_workloads() + t.BF16_EXTRA:
     t.check(w)
+for w in t.RANDOM_SMALL:
+    if w.dtype == "bf16":
+        t.check(w, rows=t._all_rows(w) if w.normalizer == "relu" else None)
 # many short work items per CTA (the ring wraps, work items are handed out by the hardware) on the forced kernel
 import torch, paper_2605_05023_b200 as pk
 from synth_inputs import Workload, make_qkv
@@ -642,21 +649,44 @@ def random_combinations(n, seed, large=False):
             kw["scale"] = float(rng.choice([0.05, 0.2, 1.0 / math.sqrt(D) * 1.7]))
         o_dtype = "fp32" if fp32 or rng.rand() < 0.3 else "bf16"
         std = float(rng.choice([1.0, 1.5]))
-        # The sigmoid normaliser does not normalise rows: with wide inputs or a growing bias |O| passes 5.12, from
-        # where on half a bf16 spacing alone exceeds the bound on O; such cases store fp32, as configuration 4(b) does.
-        if norm == "sigmoid" and (std > 1.0 or "slopes" in kw):
+        # The drawn combination is kept inside the domain in which the bounds on O and LSE mean something:
+        # (1) the sigmoid normaliser does not normalise rows: with wide inputs, a large scale or a growing bias |O|
+        # passes 5.12, from where on half a bf16 spacing alone exceeds the bound on O; such cases store fp32, as
+        # configuration 4(b) does;
+        if norm == "sigmoid" and (std > 1.0 or "slopes" in kw or "scale" in kw):
             o_dtype = "fp32"
+        # (2) the absolute bound on a bf16 O presumes V of unit scale (with N(0, 1.5^2) values a sharply peaked row
+        # returns |O| up to 7, where half a bf16 spacing is 1.6e-2 and the bf16 rounding of the dominant weight adds
+        # up to 1.3e-2); D = 256 normalises by the rounded weights and takes the wider values, as configuration 4 does;
+        if not fp32 and o_dtype == "bf16" and D < 256:
+            std = 1.0
+        # (3) fp32: a bias that grows to hundreds (slope +1 over hundreds of positions) leaves the scores with a
+        # spacing of 3e-5, above the fp32 bound whatever the kernel does, so positive slopes stay within 16 over
+        # the sequence.
+        if fp32 and "slopes" in kw and max(kw["slopes"]) > 0:
+            f = min(1.0, 16.0 / (max(kw["slopes"]) * max(sq, sk)))
+            kw["slopes"] = tuple(float(x) * f for x in kw["slopes"])
         out.append(Workload(f"{'R' if large else 'r'}{idx:02d}_{mask}_{norm}_{score}_d{D}_g{group}", B, hq, hkv, sq, sk, D,
                             dtype="fp32" if fp32 else "bf16", o_dtype=o_dtype, std=std, seed=3000 + idx, **kw))
     return out
 
 
-@pytest.mark.parametrize("w", random_combinations(96, 20261125), ids=lambda w: w.name)
+def _all_rows(w):
+    return np.arange(w.B * w.Hq * w.Sq, dtype=np.int64)
+
+
+RANDOM_SMALL = [w.with_(name=f"s{k}_{w.name}") for k, seed in enumerate((20261125, 1, 2)) for w in random_combinations(96, seed)]
+RANDOM_LARGE = [w.with_(name=f"s{k}_{w.name}") for k, seed in enumerate((20261126, 3)) for w in random_combinations(24, seed, large=True)]
+
+
+@pytest.mark.parametrize("w", RANDOM_SMALL, ids=lambda w: w.name)
 def test_seeded_random_combinations(w):
-    check(w)
+    # (ReLU: the per-row bound of `check` is conditioned on scores away from zero, which random scales do not
+    # guarantee; these cases are held to the bound relative to the largest output.)
+    check(w, rows=_all_rows(w) if w.normalizer == "relu" else None)
 
 
-@pytest.mark.parametrize("w", random_combinations(32, 20261126, large=True), ids=lambda w: w.name)
+@pytest.mark.parametrize("w", RANDOM_LARGE, ids=lambda w: w.name)
 def test_seeded_random_combinations_of_many_work_items(w):
     check(w, rows=sampled_rows(w, 24, 2, seed=sum(map(ord, w.name)), every_head=6))
 
