@@ -549,9 +549,9 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             if constexpr (kTileCap) {
                 float zmax = 0.f;
 #pragma unroll
-                for (int c = 0; c < kWgCols / 32; ++c) softcap_quad_chunk32(&y[c * 32], sc, zmax);
-                if (__any_sync(0xffffffffu, zmax > sc.zq_limit)) {
-                    // beyond the quadratic's range: the cubic (up to half the cap) or the exponential form, on the raw scores
+                for (int c = 0; c < kWgCols / 32; ++c) softcap_lin_chunk32(&y[c * 32], sc, zmax);
+                if (__any_sync(0xffffffffu, zmax > sc.zl_limit)) {
+                    // beyond the first polynomial's range: the cubic (up to half the cap) or the exponential form, on the raw scores
                     const bool exact = __any_sync(0xffffffffu, zmax > sc.z_limit);
                     ptx::tmem_ld_32x32(ts, *reinterpret_cast<uint32_t(*)[32]>(&y[0]));
                     ptx::tmem_ld_32x32(ts + 32, *reinterpret_cast<uint32_t(*)[32]>(&y[32]));

@@ -681,7 +681,7 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
                             if (!((RELU && relu_raw) || (SIGMOID && sig_raw))) score_chunk32<true>(&y[c * 32], sc, rowoff - (float)(c * 32));
                         }
                         else if constexpr (kRedo) score_chunk32_tile(&y[c * 32], sc, rowoff - (float)(c * 32), poly, zmax);
-                        else score_chunk32_quad(&y[c * 32], sc, rowoff - (float)(c * 32), zmax);
+                        else score_chunk32_lin(&y[c * 32], sc, rowoff - (float)(c * 32), zmax);
                     }
                     if (kMasked) {
                         // One bit test per element (two compares per element made partial tiles cost half as much
@@ -713,10 +713,10 @@ __device__ __forceinline__ void softmax_role(const AttnParams& p, Barriers* bars
             if constexpr (SCORE == kScoreGeneric) {
                 load_score_max(std::false_type{}, !full_tile, std::false_type{});
                 if constexpr (!SIGMOID && !RELU) {
-                    // Softcap: the first pass caps with the quadratic (scores up to 0.35 of the cap).  A score of this
+                    // Softcap: the first pass caps with a + b s^2 (scores up to 0.2 of the cap).  A score of this
                     // warp's rows beyond that (rare)?  Then the pass runs once more: with the cubic (up to half the
                     // cap), or, beyond that too, on the tile capped exactly in TMEM with the identity coefficients.
-                    if (__any_sync(0xffffffffu, zmax > sc.zq_limit)) {
+                    if (__any_sync(0xffffffffu, zmax > sc.zl_limit)) {
                         const bool exact = __any_sync(0xffffffffu, zmax > sc.z_limit);
                         if (exact) softcap_exact_in_tmem(tm + buf * kBN, kBN / 32, sc.cap_in, sc.cap_out);
                         poly = cap_poly(sc, exact);

@@ -541,23 +541,26 @@ def test_softcap_with_a_few_scores_beyond_the_polynomial_range(w):
     assert np.abs(lse.double().cpu().numpy() - lse_ref).max() <= tol_l
 
 
-# Softcap, the band between the two polynomials: the first pass over a key tile caps with a quadratic (scores up to
-# 0.35 of the cap); a warp whose tile holds a larger score repeats the pass with the cubic (up to half the cap) or, beyond
-# that, with the exponential form.  Caps chosen against the score distribution (standard deviation of scale * s: 1 at
-# std = 1, 2.25 at std = 1.5) so that most warp tiles have their largest score inside the band, some below it and some
-# above: all three paths inside one launch, with a fixed reference, a running maximum and a position bias.
+# Softcap, the band between the two polynomials: the first pass over a key tile caps with a + b s^2 (scores up to
+# 0.2 of the cap); a warp whose tile holds a larger score repeats the pass with the cubic in s^2 (up to half the cap) or,
+# beyond that, with the exponential form.  Caps chosen against the score distribution (standard deviation of scale * s:
+# 1 at std = 1, 2.25 at std = 1.5): with the small caps most warp tiles have their largest score inside the band and
+# some above it, with the two larger ones (the largest of a warp tile's 4096 scores sits near 0.2 of the cap) some
+# tiles stay with the first pass and some repeat it; with a fixed reference, a running maximum and a position bias.
 @pytest.mark.parametrize("w", [
     Workload("cap_band_d128", 1, 2, 2, 900, 900, 128, seed=180, causal=True, softcap=9.0),
     Workload("cap_band_d128_alibi", 1, 2, 1, 900, 900, 128, seed=181, causal=True, softcap=9.0, slopes=(-0.25, -0.0625)),
     Workload("cap_band_d64", 1, 2, 2, 700, 700, 64, seed=182, softcap=9.0),
     Workload("cap_band_d256_fixed_reference", 1, 2, 2, 640, 640, 256, seed=183, causal=True, softcap=20.0, std=1.5),
     Workload("cap_band_d256_running_max", 1, 2, 1, 640, 640, 256, seed=184, causal=True, softcap=20.0, slopes=(-0.5, 0.25), std=1.5),
+    Workload("cap_edge_d128", 1, 2, 2, 900, 900, 128, seed=185, causal=True, softcap=17.0),
+    Workload("cap_edge_d256", 1, 2, 2, 640, 640, 256, seed=186, causal=True, softcap=40.0, std=1.5),
 ], ids=lambda w: w.name)
 def test_softcap_scores_between_the_two_polynomial_ranges(w):
     q, k, v = make_qkv(w)
     raw = torch.einsum("bhid,bhjd->bhij", q.float()[:, ::w.Hq // w.Hkv], k.float()) * (w.scale or w.D ** -0.5)
     x = raw.abs() / w.softcap
-    band = float(((x > 0.35) & (x <= 0.5)).float().mean())
+    band = float(((x > 0.2) & (x <= 0.5)).float().mean())
     beyond = float((x > 0.5).float().mean())
     assert band > 2e-4 and beyond < band, f"{w.name}: band {band:.5f}, beyond {beyond:.5f}"
     check(w)
