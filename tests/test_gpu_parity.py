@@ -579,6 +579,13 @@ LONG_CASES = [
     Workload("long_docs_d128", 1, 2, 1, 65536, 65536, 128, seed=153, causal=True,
              cu_seqlens=(0, 5000, 5001, 30000, 30130, 65536)),
     Workload("long_cross", 1, 2, 2, 300, 65536, 64, seed=154),
+    # more heads than one L2 section of the work order holds (two sections, handed out as one under a document mask),
+    # with and without global tokens
+    Workload("sections_share_question", 1, 16, 16, 8192, 8192, 128, seed=155, causal=True,
+             cu_seqlens=(0, 4096, 5120, 6144, 7168, 8192), global_len=4096),
+    Workload("sections_docs_test_query", 1, 16, 16, 8192, 8192, 128, seed=156, causal=True,
+             cu_seqlens=(0, 1000, 3000, 3001, 6500, 7168, 8192), test_query_start=7168),
+    Workload("sections_global_window", 1, 24, 24, 8192, 8192, 128, seed=157, window_left=64, window_right=64, global_len=128),
 ]
 
 
