@@ -181,24 +181,34 @@ __device__ __forceinline__ void work_order_front(int lin, int units_total, int s
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-// How many query blocks of every head hold a global token's row under a non-causal two-sided window (Global Sliding
-// Window, Appendix A.2): such a row sees every key, so its block's work item is the longest of its head by far, and
-// handed out section by section the last section's long items can end the grid on a few SMs.  They open the work
-// order instead, when that helps: 0 under a causal mask (it bounds those rows like the others), without global
-// tokens, when the long items have fewer than four times the key tiles of the window items, when a section lasts
-// longer than a long item anyway (then the long items of the last section are hidden in it, and section order keeps
-// its K and V in L2), or when more than a quarter of the blocks would qualify.  `sec_units`: work-order units
-// ((batch, head) or head pairs) per section; `workers`: CTAs that run at once.
+// How many query blocks of every head open the work order, ahead of the sections: blocks whose work items are the
+// longest of their head by far, which, handed out section by section, can end the grid on a few SMs when the last
+// section starts late.  Two cases.  (a) Global Sliding Window (Appendix A.2), non-causal two-sided window: the blocks
+// that hold a global token's row (such a row sees every key, the others a window).  (b) The causal blockwise mask with
+// its test-query clause: the blocks of the test query's rows (they see every key up to their own position, the
+// others their own document).  0 when there is little to gain: the long items have fewer than four times the key tiles
+// of the others (for documents, estimated from the mean document length), a section lasts longer than a long item
+// anyway (then the long items of the last section are hidden in it, and section order keeps its K and V in L2), or
+// more than a quarter of the blocks would qualify.  `sec_units`: work-order units ((batch, head) or head pairs) per
+// section; `workers`: CTAs that run at once.
 inline int leading_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long sec_units, int workers) {
-    if (!(p.mask_flags & kMaskGlobal) || (p.mask_flags & kMaskCausal) || nqb < 4) return 0;
-    if (!(p.mask_flags & kMaskWindow) || p.window_left < 0 || p.window_right < 0) return 0;
-    const long long window_tiles = ((long long)p.window_left + p.window_right + rows) / key_tile + 2;
+    if (nqb < 4) return 0;
+    long long light_tiles, long_rows;
+    if ((p.mask_flags & kMaskGlobal) && !(p.mask_flags & kMaskCausal)) {
+        if (!(p.mask_flags & kMaskWindow) || p.window_left < 0 || p.window_right < 0) return 0;
+        light_tiles = ((long long)p.window_left + p.window_right + rows) / key_tile + 2;
+        long_rows = std::min<long long>(std::max<long long>((long long)p.global_len - (p.Sk - p.Sq), 0), p.Sq);
+    } else if ((p.mask_flags & kMaskTestQuery) && (p.mask_flags & kMaskCausal) && !(p.mask_flags & kMaskGlobal)) {
+        light_tiles = ((long long)p.Sk / std::max(p.num_docs, 1) + rows) / key_tile / 2 + 2;
+        long_rows = std::max<long long>((long long)p.Sq - p.test_query_start, 0);
+    } else {
+        return 0;
+    }
     const long long long_tiles = (long long)p.Sk / key_tile;
-    if (long_tiles < 4 * window_tiles) return 0;
-    const long long global_rows = std::min<long long>(std::max<long long>((long long)p.global_len - (p.Sk - p.Sq), 0), p.Sq);
-    const int blocks = (int)((global_rows + rows - 1) / rows);
-    if (blocks * 4 > nqb) return 0;
-    const long long section_steps = sec_units * (blocks * long_tiles + (nqb - blocks) * window_tiles) / std::max(workers, 1);
+    if (long_tiles < 4 * light_tiles) return 0;
+    const int blocks = (int)((long_rows + rows - 1) / rows);
+    if (blocks == 0 || blocks * 4 > nqb) return 0;
+    const long long section_steps = sec_units * (blocks * long_tiles + (nqb - blocks) * light_tiles) / std::max(workers, 1);
     return (section_steps >= long_tiles) ? 0 : blocks;
 }
 

@@ -214,7 +214,7 @@ __device__ __forceinline__ ItemG decode_item(const AttnParams& p, int lin, const
     it.slope[0] = p.slopes ? __ldg(p.slopes + it.ht[0]) : 0.f;
     it.slope[1] = p.slopes ? __ldg(p.slopes + it.ht[1]) : 0.f;
     it.rev_top = -1;
-    if (!(p.mask_flags & kMaskGlobal) && (it.slope[0] < 0.f || it.slope[1] < 0.f)) {
+    if (!GLB && !(p.mask_flags & kMaskGlobal) && (it.slope[0] < 0.f || it.slope[1] < 0.f)) {   // (the global-token instances walk by position only)
         // walk the key tiles downwards: tile j becomes position (top - j)
         int top = 0;
 #pragma unroll
@@ -1008,6 +1008,30 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_cons
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+// Heads per section of the work order: as many KV heads as keep the section's K and V within about 40 MB of L2, in
+// equal sections, whole GQA groups.
+inline long long section_heads(const AttnParams& p) {
+    const long long kv_bytes = 2ll * p.Sk * p.D * 2;
+    long long kv_heads = (40ll << 20) / kv_bytes;
+    if (kv_heads < 1) kv_heads = 1;
+    const long long bh = (long long)p.B * p.Hq;
+    long long sec_max = kv_heads * p.group;
+    if (sec_max > bh) sec_max = bh;
+    const long long n_sec = (bh + sec_max - 1) / sec_max;
+    long long sec = (bh + n_sec - 1) / n_sec;
+    return (sec + p.group - 1) / p.group * p.group;
+}
+// Query blocks per head that open the work order (leading_blocks in attn_params.cuh) when the call runs on the
+// global-token instances, the ones that decode such an order: work items of two heads x 128 rows with an even GQA
+// group, else one head x 256 rows; the weight-ordered list must cover the blocks (those instances: 1024).
+inline int planned_leading_blocks(const AttnParams& p) {
+    const int units = (p.group % 2 == 0) ? 2 : 1;
+    const long long rows = (units == 2) ? kBM : 2 * kBM;
+    const long long nqb = (p.Sq + rows - 1) / rows;
+    if (nqb > Cfg<128, 2, false>::kMaxOrdered) return 0;
+    return leading_blocks(p, (int)rows, kBN, (int)nqb, section_heads(p) / units, device_sm_count());
+}
+
 template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>
 int launch_instance(AttnParams p, cudaStream_t stream) {
     using C = Cfg<D, NQ, TMA_OUT>;
@@ -1025,15 +1049,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     else if (!make_map(&mo, p.o, p.B, p.Hq, p.Sq, D, p.os, 32, 32, 64)) return ATTN_ERR_CUDA;
     // Heads per section of the work order: as many KV heads as keep the section's K and V within
     // about 40 MB of L2, in equal sections, whole GQA groups.
-    const long long kv_bytes = 2ll * p.Sk * D * 2;
-    long long kv_heads = (40ll << 20) / kv_bytes;
-    if (kv_heads < 1) kv_heads = 1;
     const long long bh = (long long)p.B * p.Hq;
-    long long sec_max = kv_heads * p.group;
-    if (sec_max > bh) sec_max = bh;
-    const long long n_sec = (bh + sec_max - 1) / sec_max;
-    long long sec = (bh + n_sec - 1) / n_sec;
-    sec = (sec + p.group - 1) / p.group * p.group;
+    const long long sec = section_heads(p);
     p.sec_heads = (int)sec;
     // Work items: two heads x 128 rows with an even GQA group, else one head x 256 rows (see decode_item).
     p.head_pair = (p.group % 2 == 0) ? 1 : 0;
@@ -1050,7 +1067,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
         const long long sections = (units + sec_units - 1) / sec_units;
         p.sec_merge_from = ((p.mask_flags & kMaskDocument) && sections >= 2) ? (int)(sections - 2) : 0x7fffffff;
     }
-    p.front_blocks = (GLB && nqb <= C::kMaxOrdered) ? leading_blocks(p, (int)rows, kBN, (int)nqb, sec / (p.head_pair ? 2 : 1), device_sm_count()) : 0;
+    // (the leading blocks are the first of the weight-ordered list; only the global-token instances decode them)
+    p.front_blocks = GLB ? planned_leading_blocks(p) : 0;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }
