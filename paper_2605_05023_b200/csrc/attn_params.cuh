@@ -190,8 +190,8 @@ __device__ __forceinline__ void work_order_front(int lin, int units_total, int s
 // of the others (for documents, estimated from the mean document length), a section lasts longer than a long item
 // anyway (then the long items of the last section are hidden in it, and section order keeps its K and V in L2), or
 // more than a quarter of the blocks would qualify.  `sec_units`: work-order units ((batch, head) or head pairs) per
-// section; `workers`: CTAs that run at once.
-inline int leading_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long sec_units, int workers) {
+// section, `units_total`: all of them; `workers`: CTAs that run at once.
+inline int leading_blocks(const AttnParams& p, int rows, int key_tile, int nqb, long long sec_units, long long units_total, int workers) {
     if (nqb < 4) return 0;
     long long light_tiles, long_rows;
     if ((p.mask_flags & kMaskGlobal) && !(p.mask_flags & kMaskCausal)) {
@@ -199,6 +199,7 @@ inline int leading_blocks(const AttnParams& p, int rows, int key_tile, int nqb, 
         light_tiles = ((long long)p.window_left + p.window_right + rows) / key_tile + 2;
         long_rows = std::min<long long>(std::max<long long>((long long)p.global_len - (p.Sk - p.Sq), 0), p.Sq);
     } else if ((p.mask_flags & kMaskTestQuery) && (p.mask_flags & kMaskCausal) && !(p.mask_flags & kMaskGlobal)) {
+        if (units_total <= 2 * sec_units) return 0;      // one section after the merge of the last two: the long blocks lead it anyway
         light_tiles = ((long long)p.Sk / std::max(p.num_docs, 1) + rows) / key_tile / 2 + 2;
         long_rows = std::max<long long>((long long)p.Sq - p.test_query_start, 0);
     } else {

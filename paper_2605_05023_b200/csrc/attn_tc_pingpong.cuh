@@ -1029,7 +1029,7 @@ inline int planned_leading_blocks(const AttnParams& p) {
     const long long rows = (units == 2) ? kBM : 2 * kBM;
     const long long nqb = (p.Sq + rows - 1) / rows;
     if (nqb > Cfg<128, 2, false>::kMaxOrdered) return 0;
-    return leading_blocks(p, (int)rows, kBN, (int)nqb, section_heads(p) / units, device_sm_count());
+    return leading_blocks(p, (int)rows, kBN, (int)nqb, section_heads(p) / units, (long long)p.B * p.Hq / units, device_sm_count());
 }
 
 template <int D, int NQ, int SCORE, int NORM, bool GLB, bool TMA_OUT>

@@ -727,7 +727,8 @@ int launch_instance(AttnParams p, cudaStream_t stream) {
     const long long nqb = (p.Sq + kBM - 1) / kBM;
     const long long grid = nqb * bh;
     if (grid > 0x7fffffffLL) return ATTN_ERR_SHAPE;
-    p.front_blocks = leading_blocks(p, kBM, kBN, (int)nqb, sec, device_sm_count());
+    // (global tokens only: their rows are the first blocks; this kernel's order already starts a section with the last blocks)
+    p.front_blocks = (p.mask_flags & kMaskGlobal) ? leading_blocks(p, kBM, kBN, (int)nqb, sec, bh, device_sm_count()) : 0;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, p);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_CUDA;
 }

@@ -586,14 +586,17 @@ LONG_CASES = [
     Workload("sections_docs_test_query", 1, 16, 16, 8192, 8192, 128, seed=156, causal=True,
              cu_seqlens=(0, 1000, 3000, 3001, 6500, 7168, 8192), test_query_start=7168),
     Workload("sections_global_window", 1, 24, 24, 8192, 8192, 128, seed=157, window_left=64, window_right=64, global_len=128),
-    # causal blockwise masks whose test-query blocks open the work order (these calls run on the global-token
-    # instances): 256-row items, two-head items with a bias, several sections
+    # causal blockwise masks with a test query: one or two sections (plain instances), and three sections, where the
+    # test-query blocks open the work order and the call runs on the global-token instances (256-row items; two-head
+    # items with a bias)
     Workload("test_query_leads", 1, 3, 3, 4096, 4096, 128, seed=158, causal=True,
              cu_seqlens=tuple(range(0, 4097, 512)), test_query_start=3584),
     Workload("test_query_leads_pair_alibi", 1, 4, 2, 4096, 4096, 64, seed=159, causal=True, slopes=alibi_slopes(4),
              cu_seqlens=(0, 300, 1100, 1101, 2048, 3000, 3584, 4096), test_query_start=3500),
     Workload("test_query_leads_sections", 1, 24, 24, 8192, 8192, 128, seed=160, causal=True,
              cu_seqlens=tuple(range(0, 8193, 1024)), test_query_start=7168),
+    Workload("test_query_leads_sections_pair_alibi", 1, 24, 12, 16384, 16384, 128, seed=161, causal=True,
+             slopes=alibi_slopes(24), cu_seqlens=tuple(range(0, 16385, 2048)), test_query_start=14336),
 ]
 
 
